@@ -1,0 +1,242 @@
+"""Pins for the oracle's Residual Activation Compensation, routing and MoE
+forward: the paper's shrink inequality and sign convention, monotone error over
+the paper's channel ratios, the two degenerate ratios, brute force on tiny
+inputs, a float64 triple loop written independently of numpy's matmul, the
+exact-integer special case, linearity and the dense special case."""
+import os
+
+import numpy as np
+import torch
+
+from oracle import formats as F
+from oracle import moe as M
+from oracle import nvfp4 as Q
+from oracle import rac as R
+from paper_2607_15810_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _ratios():
+    with open(os.path.join(GOLD, "rac_ratios.txt")) as fh:
+        line = [ln for ln in fh if not ln.startswith("#") and ln.strip()][0]
+    return [float(v) for v in line.split()]
+
+
+def _dense():
+    x, w = synth.dense_inputs(seed=0)
+    return x.to(torch.float32).numpy(), w.to(torch.float32).numpy()
+
+
+def test_shrink_inequality_and_sign_for_both_residual_scale_readings():
+    x, _ = _dense()
+    for r_gs in (None, "own"):
+        plain = R.rac(x, 0, None, r_gs)
+        e0 = np.linalg.norm(R.reconstruct_real(plain) - x)
+        assert e0 == np.linalg.norm(Q.dequantize_real(plain["codes"], plain["sf"], plain["gs"]) - x)
+        prev = e0
+        for pct in _ratios():
+            n_sel = int(round(x.shape[1] * pct / 100))
+            site = R.rac(x, n_sel, None, r_gs)
+            e = np.linalg.norm(R.reconstruct_real(site) - x)
+            assert e < prev, (r_gs, pct, e, prev)           # strictly shrinking, Eq. residual-shrink
+            prev = e
+            # the opposite sign would grow the error
+            wrong = (Q.dequantize_real(site["codes"], site["sf"], site["gs"])
+                     + Q.dequantize_real(site["r_codes"], site["r_sf"], site["r_gs"]))
+            assert np.linalg.norm(wrong - x) > e0
+
+
+def test_degenerate_ratios():
+    x, _ = _dense()
+    K = x.shape[1]
+    s0 = R.rac(x, 0)
+    assert s0["sel"].size == 0 and not s0["r_codes"].any()
+    sK = R.rac(x, K)
+    assert np.array_equal(sK["sel"], np.arange(K))
+    full_c, full_s, _ = Q.quantize(sK["residual"], sK["r_gs"])
+    assert np.array_equal(sK["r_codes"], full_c) and np.array_equal(sK["r_sf"], full_s)
+    # masking never touches the scales
+    s16 = R.rac(x, 16)
+    assert np.array_equal(s16["r_sf"], full_s)
+    keep = np.zeros(K, bool)
+    keep[s16["sel"]] = True
+    assert np.array_equal(s16["r_codes"][:, keep], full_c[:, keep])
+    assert not s16["r_codes"][:, ~keep].any()
+
+
+def test_selection_is_brute_force_topk_with_low_index_ties():
+    scores = np.array([3.0, 7.0, 7.0, 1.0, 9.0, 7.0, 0.0, 3.0])
+    for n in range(9):
+        # brute force: repeatedly take the largest remaining score, lowest index first
+        rest, chosen = list(range(8)), []
+        for _ in range(n):
+            best = max(rest, key=lambda j: (scores[j], -j))
+            chosen.append(best)
+            rest.remove(best)
+        assert list(R.select_channels(scores, n)) == sorted(chosen)
+    x, _ = _dense()
+    site = R.rac(x[:9, :32], 5)
+    r = site["residual"].astype(np.float64)
+    brute = sorted(sorted(range(32), key=lambda j: (-float((r[:, j] ** 2).sum()), j))[:5])
+    assert list(site["sel"]) == brute
+    assert np.allclose(site["scores"], [(r[:, j] ** 2).sum() for j in range(32)], rtol=1e-12)
+
+
+def test_dense_config_selects_inside_the_outlier_blocks():
+    """The x20 outlier channels inflate their 16-block's scale, so every channel
+    of those four blocks carries a large residual: the paper's "vertical bands"
+    (Section "Activation Error Compensation for Rollout-side")."""
+    x, _ = _dense()
+    site = R.rac(x, 16)
+    blocks = {c // 16 for c in synth.DENSE_OUTLIER_CHANNELS}
+    assert {int(j) // 16 for j in site["sel"]} <= blocks
+    # the residual really is Q_A(X) - X (Eq. residual-def), not X - Q_A(X)
+    xh = Q.dequantize_f32(site["codes"], site["sf"], site["gs"])
+    assert np.array_equal(site["residual"], xh - x)
+
+
+def test_routing_against_brute_force():
+    rng = np.random.default_rng(5)
+    logits = rng.normal(size=(13, 6)).astype(np.float32)
+    logits[2, 1] = logits[2, 4] = logits[2].max() + 1       # a tie at the top
+    ids, w = M.route(logits, 3, renormalize=True)
+    for t in range(13):
+        order = sorted(range(6), key=lambda e: (-float(logits[t, e]), e))[:3]
+        assert list(ids[t]) == order
+        p = np.exp(logits[t].astype(np.float64))
+        p /= p.sum()
+        want = p[order] / p[order].sum()
+        assert np.allclose(w[t], want, rtol=1e-6)
+    ids2, w2 = M.route(logits, 3, renormalize=False)
+    assert np.array_equal(ids, ids2)
+    assert np.all(w2.sum(axis=1) < 1)
+    counts, offsets, perm = M.dispatch(ids, 6)
+    assert counts.sum() == 13 * 3 and offsets[0] == 0 and offsets[-1] == 39
+    assert np.all(np.diff(offsets) == counts)
+    assert sorted(perm) == list(range(39))
+    keys = [(int(ids.reshape(-1)[p]), int(p)) for p in perm]
+    assert keys == sorted(keys)                              # (expert, token, slot) order
+
+
+def _tiny_weights(n, N, K, seed, std=0.05):
+    w = (torch.randn(n, N, K, generator=torch.Generator().manual_seed(seed)) * std)
+    w = w.to(torch.bfloat16).to(torch.float32).numpy()
+    _, q, sf, gs = Q.fake_quant_weights(w)
+    return dict(codes=F.unpack_nibbles(q), sf=sf, gs=gs)
+
+
+def _triple_loop(a, b):
+    """a [M,K], b [N,K] -> a b^T with python floats (IEEE double), no numpy matmul."""
+    out = [[0.0] * len(b) for _ in a]
+    for i, ar in enumerate(a):
+        for j, br in enumerate(b):
+            s = 0.0
+            for u, v in zip(ar, br):
+                s += u * v
+            out[i][j] = s
+    return np.array(out)
+
+
+def _scalar_dequant(codes, sf8, gs):
+    """Element-by-element dequantization written from the format definition."""
+    e2 = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    out = np.zeros(codes.shape)
+    for i in range(codes.shape[0]):
+        for k in range(codes.shape[1]):
+            c = int(codes[i, k])
+            s = int(sf8[i, k // 16])
+            ef, m = s >> 3, s & 7
+            sc = (m / 8.0) * 2.0 ** -6 if ef == 0 else (1 + m / 8.0) * 2.0 ** (ef - 7)
+            out[i, k] = (-1.0 if c & 8 else 1.0) * e2[c & 7] * sc * float(gs)
+    return out
+
+
+def test_dense_gemm_against_triple_loop_and_linearity():
+    x, w = synth.dense_inputs(seed=3, T=5, K=32, N=4, outlier_channels=(3,))
+    x = x.to(torch.float32).numpy()
+    wq = _tiny_weights(1, 4, 32, 9)
+    res = M.dense_w4a4_rac(x, wq["codes"][0], wq["sf"][0], wq["gs"][0], n_sel=8)
+    site = res["site"]
+    xa = _scalar_dequant(site["codes"], site["sf"], site["gs"])
+    ra = _scalar_dequant(site["r_codes"], site["r_sf"], site["r_gs"])
+    wa = _scalar_dequant(wq["codes"][0], wq["sf"][0], wq["gs"][0])
+    want = _triple_loop((xa - ra).tolist(), wa.tolist())
+    assert np.allclose(res["y64"], want, rtol=1e-12, atol=1e-15)
+    # linearity: W X~ = W Q(X) - W (M (.) Q(dX))
+    lin = _triple_loop(xa.tolist(), wa.tolist()) - _triple_loop(ra.tolist(), wa.tolist())
+    assert np.allclose(res["y64"], lin, rtol=1e-10, atol=1e-14)
+    # n_sel = 0 is the plain W4A4 product
+    plain = M.dense_w4a4_rac(x, wq["codes"][0], wq["sf"][0], wq["gs"][0], n_sel=0)
+    assert np.allclose(plain["y64"], _triple_loop(xa.tolist(), wa.tolist()), rtol=1e-12, atol=1e-15)
+    absd = _triple_loop((np.abs(xa) + np.abs(ra)).tolist(), np.abs(wa).tolist())
+    assert np.allclose(res["absdot"], absd, rtol=1e-12)
+
+
+def test_exact_integer_special_case():
+    """Scales of one and integer-valued codes: the contraction is a small-integer
+    matrix product (textbook check, exact)."""
+    rng = np.random.default_rng(11)
+    ints = np.array([0, 1, 2, 3, 4, 6, -1, -2, -3, -4, -6])
+    a = rng.choice(ints, (6, 32)).astype(np.float32)
+    a[:, 0] = 6
+    a[:, 16] = -6
+    b = rng.choice(ints, (3, 32)).astype(np.float32)
+    b[:, 0] = 6
+    b[:, 16] = 6
+    ca, sa, ga = Q.quantize(a, np.float32(1.0))
+    cb, sb, gb = Q.quantize(b, np.float32(1.0))
+    assert np.all(sa == 0x38) and np.all(sb == 0x38)        # E4M3 code of 1.0
+    res = M.dense_w4a4_rac(a, cb, sb, gb, n_sel=0, a_gs=np.float32(1.0))
+    assert np.array_equal(res["y64"], (a.astype(np.int64) @ b.astype(np.int64).T).astype(np.float64))
+
+
+def test_moe_single_expert_reduces_to_dense_and_matches_loops():
+    shape = synth.MoEShape("t", 21, 6, 32, 1, 1, 16, 0.05, 1, 3.0, 10.0)
+    x, _ = synth.activations(shape)
+    x = x.to(torch.float32).numpy()
+    logits = np.zeros((6, 1), np.float32)
+    w13 = _tiny_weights(1, 32, 32, 31)
+    w2 = _tiny_weights(1, 32, 16, 32)
+    a2_gs = np.float32(0.002)
+    out = M.moe_forward(x, logits, w13, w2, 1, 8, 4, a2_gs)
+    assert np.array_equal(out["perm"], np.arange(6)) and np.all(out["weights"] == 1.0)
+    d = M.dense_w4a4_rac(x, w13["codes"][0], w13["sf"][0], w13["gs"][0], n_sel=8)
+    assert np.array_equal(out["g64"], d["y64"])
+    g = out["g64"]
+    h = np.array([[(gi / (1 + np.exp(-gi))) * ui for gi, ui in zip(row[:16], row[16:])] for row in g])
+    assert np.allclose(out["h64"], h, rtol=1e-13)
+    d2 = M.dense_w4a4_rac(out["h"], w2["codes"][0], w2["sf"][0], w2["gs"][0], n_sel=4, a_gs=a2_gs)
+    assert np.array_equal(out["out64"], d2["y64"])
+
+
+def test_moe_two_experts_against_explicit_loops():
+    shape = synth.MoEShape("t", 22, 9, 32, 3, 2, 16, 0.05, 1, 3.0, 10.0)
+    x, _ = synth.activations(shape)
+    x = x.to(torch.float32).numpy()
+    logits = synth.router_logits(shape).numpy()
+    w13 = _tiny_weights(3, 32, 32, 41)
+    w2 = _tiny_weights(3, 32, 16, 42)
+    a2_gs = np.float32(0.003)
+    out = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2_gs, renormalize=True)
+    # re-derive the output token by token from the exported intermediates
+    xt = R.reconstruct_real(out["site13"])
+    ht = R.reconstruct_real(out["site2"])
+    inv = np.empty(18, int)
+    inv[out["perm"]] = np.arange(18)
+    want = np.zeros((9, 32))
+    for t in range(9):
+        for s in range(2):
+            e = int(out["ids"][t, s])
+            row = inv[t * 2 + s]
+            assert out["offsets"][e] <= row < out["offsets"][e + 1]
+            w13e = _scalar_dequant(w13["codes"][e], w13["sf"][e], w13["gs"][e])
+            g = _triple_loop([xt[t].tolist()], w13e.tolist())[0]
+            assert np.allclose(out["g64"][row], g, rtol=1e-12, atol=1e-15)
+            w2e = _scalar_dequant(w2["codes"][e], w2["sf"][e], w2["gs"][e])
+            y = _triple_loop([ht[row].tolist()], w2e.tolist())[0]
+            want[t] += float(out["weights"][t, s]) * y
+    assert np.allclose(out["out64"], want, rtol=1e-11, atol=1e-14)
+    assert np.array_equal(out["out"], F.bf16_round(out["out64"]))
+    # site-2 statistics run over all dispatched rows at once
+    assert out["site2"]["codes"].shape == (18, 16) and out["site2"]["sel"].size == 8

@@ -1,0 +1,179 @@
+/*
+ * quads.h -- C ABI of the B200 (sm_100a) NVFP4 MoE rollout forward and the
+ * trainer-side weight fake-quant.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the comment says "host".  The args
+ *     struct and the returned strings are host memory.
+ *   - The caller owns every buffer.  The library never allocates or frees
+ *     device memory; scratch comes from the `workspace` argument, whose
+ *     minimum size the matching *_workspace_bytes() function returns.
+ *     Workspaces must be 256-byte aligned.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) and the call returns without synchronising.
+ *   - Argument errors are detected on the host and returned before anything is
+ *     launched.  A CUDA launch error is returned as QUADS_ERR_CUDA.  A device
+ *     wait that ran out of its iteration budget is recorded in the workspace and
+ *     can be read with quads_moe_async_status() after the stream is synchronised.
+ *   - Inputs must be finite.  K (and H, I) must be multiples of 16 for the
+ *     quantizers and multiples of 128 for GEMM operands.
+ *
+ * NVFP4 format (paper, Section "Low-Precision Inference", paragraph FP4):
+ * E2M1 elements {0,0.5,1,1.5,2,3,4,6} per sign; 16 consecutive elements along
+ * the contraction dimension share one E4M3 scale; one FP32 per-tensor scale.
+ * Element 2i sits in the low nibble and 2i+1 in the high nibble of byte i.
+ * Scale derivation (all float32, in this order):
+ *   s_g = amax(tensor) / 2688  (1 for an all-zero tensor)
+ *   sf  = E4M3_rne_sat( amax(block) / (6 * s_g) ),  d = sf * s_g
+ *   code = E2M1_rne_sat( x * (1 / d) )   (all-zero codes when sf == 0)
+ *   dequantized value = value(code) * d
+ */
+#ifndef QUADS_H_
+#define QUADS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t quads_status;
+
+enum {
+  QUADS_OK = 0,
+  QUADS_ERR_NULL = -1,       /* a required pointer is NULL */
+  QUADS_ERR_SHAPE = -2,      /* a size breaks a divisibility or range rule */
+  QUADS_ERR_WORKSPACE = -3,  /* workspace missing, misaligned or too small */
+  QUADS_ERR_ARCH = -4,       /* the current device is not sm_100 */
+  QUADS_ERR_CUDA = -5,       /* a CUDA runtime / driver call failed */
+  QUADS_ERR_TIMEOUT = -6     /* a bounded device-side wait gave up */
+};
+
+enum {
+  QUADS_SF_LINEAR = 0, /* scale bytes as [rows, K/16], row-major (the parity layout) */
+  QUADS_SF_TILED = 1   /* 512-byte atoms of 128 rows x 4 blocks for the tensor-core path:
+                          atom (row/128, blk/4) at ((row/128) * ceil(K/64) + blk/4) * 512,
+                          byte (row%32)*16 + ((row%128)/32)*4 + blk%4 inside it; rows are
+                          padded to a multiple of 128 and K to a multiple of 64 */
+};
+
+/* Human-readable name of a status code (host string, never NULL). */
+const char* quads_status_string(quads_status s);
+
+/* Bytes of a QUADS_SF_TILED scale buffer for one [rows, K] tensor. */
+size_t quads_sf_tiled_bytes(int64_t rows, int64_t K);
+
+/*
+ * (1) Online NVFP4 activation quantization, the operator Q_A of
+ * Eq. "act-error-def" (Section "Methods"), format as in Section "Low-Precision
+ * Inference", paragraph FP4.
+ *   x      bf16 [rows, K], row stride `ld` elements (ld >= K, ld % 16 == 0),
+ *          32-byte aligned
+ *   gs_in  float[1] per-tensor scale, or NULL: amax(x)/2688 computed on device
+ *   q      out, u8 [rows, K/2]
+ *   sf     out, u8, layout per `sf_layout` ([rows, K/16] when linear)
+ *   gs_out out, float[1]: the per-tensor scale that was used (may be NULL)
+ *   workspace  >= quads_quantize_workspace_bytes() bytes
+ * rows == 0 is allowed (nothing is written except gs_out = 1 when gs_in is NULL).
+ */
+quads_status quads_quantize_nvfp4(const void* x, int64_t rows, int64_t K, int64_t ld,
+                                  const float* gs_in, uint8_t* q, uint8_t* sf, float* gs_out,
+                                  int sf_layout, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream);
+size_t quads_quantize_workspace_bytes(void);
+
+/*
+ * (4) Trainer-side Asymmetric-QAT weight fake-quant QDQ_W (Eq. "w4a16-qat-forward")
+ * and the pack for rollout weight sync (Eqs. "weight-sync", "weight-qdq-align"):
+ * one quantization decides both outputs, so the bf16 the trainer multiplies by
+ * equals, bit for bit, the bf16 dequantization of the bytes the rollout loads.
+ *   w       bf16 [n_tensors, N, K], K contiguous; every [N, K] slice is one tensor
+ *           with its own per-tensor scale
+ *   w_fq    out, bf16 [n_tensors, N, K]  (NULL to skip)
+ *   q       out, u8 [n_tensors, N, K/2]  (NULL to skip)
+ *   sf      out, u8 per `sf_layout`, one [N, K/16] (or tiled) block per tensor (NULL to skip)
+ *   gs      out, float [n_tensors] (required)
+ *   workspace >= quads_fake_quant_workspace_bytes(n_tensors) bytes
+ */
+quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t N, int64_t K,
+                                      void* w_fq, uint8_t* q, uint8_t* sf, float* gs,
+                                      int sf_layout, void* workspace, size_t workspace_bytes,
+                                      void* cuda_stream);
+size_t quads_fake_quant_workspace_bytes(int64_t n_tensors);
+
+/*
+ * (2)+(3) MoE expert layer forward with native W4A4 grouped GEMMs and Residual
+ * Activation Compensation (Section "Activation Error Compensation for
+ * Rollout-side", Eqs. "residual-def", "residual-recon", "channel-score",
+ * "channel-select"):
+ *   X~ = Q_A(X) - M_S (.) Q_A(Q_A(X) - X),  S = the n_sel channels with the
+ *   largest residual L2 norm over the current token batch,
+ * evaluated as  W X~ = W Q_A(X) - W (M_S (.) Q_A(dX)), two W4A4 tensor-core
+ * products into one accumulator (the residual shares the per-tensor scale of
+ * its activation).  Per token: top-k experts by router logit (ties to the lower
+ * id), weights = softmax over all experts restricted to the chosen ones
+ * (renormalised when `renormalize`), h = silu(W1 x) * (W3 x) rounded to bf16,
+ * requantized with `a2_gs`, out = sum_k weight_k * W2 h~.
+ *
+ * Dense mode (I == 0): one projection out[T, N] = W X~ with E = topk = 1, the
+ * weight in w13_*, no routing, no SwiGLU ("single dense W4A4+RAC GEMM").
+ *
+ * Weight buffers are exactly what quads_fake_quant_weights() writes with
+ * QUADS_SF_TILED: w13 is [E, 2I, H] (gate rows first, then up rows), w2 is
+ * [E, H, I]; H % 128 == 0, I % 128 == 0 (dense: N % 128 == 0).
+ */
+typedef struct {
+  int32_t T, H, I, E, topk;
+  int32_t N;                    /* dense mode only */
+  const void* x;                /* bf16 [T, H] */
+  const float* router_logits;   /* float [T, E]; ignored in dense mode */
+  const uint8_t* w13_q;         /* u8 [E, 2I, H/2]  (dense: [N, H/2]) */
+  const uint8_t* w13_sf;        /* tiled, E blocks of quads_sf_tiled_bytes(2I, H) */
+  const float* w13_gs;          /* float [E] */
+  const uint8_t* w2_q;          /* u8 [E, H, I/2] */
+  const uint8_t* w2_sf;         /* tiled, E blocks of quads_sf_tiled_bytes(H, I) */
+  const float* w2_gs;           /* float [E] */
+  int32_t rac_nsel_13;          /* channels compensated at the W13 input, 0..H */
+  int32_t rac_nsel_2;           /* channels compensated at the W2 input, 0..I */
+  const float* a13_gs;          /* float[1] per-tensor scale of x, NULL: amax-derived on device */
+  const float* a2_gs;           /* float[1] per-tensor scale of h; required when I > 0 */
+  int32_t renormalize;
+  void* out;                    /* bf16 [T, H]  (dense: [T, N]) */
+  /* Optional exports for verification; each may be NULL. Dispatch order means
+     assignments (token, slot) sorted by (expert, token, slot); A = T * topk. */
+  int32_t* topk_ids;            /* [T, topk] */
+  float* topk_w;                /* [T, topk] */
+  int32_t* expert_offsets;      /* [E + 1] */
+  int32_t* perm;                /* [A] flat assignment index t*topk+slot per dispatched row */
+  uint8_t* xq;                  /* [T, H/2]  Q_A(x) codes, token order */
+  uint8_t* xsf;                 /* [T, H/16] linear */
+  uint8_t* rq;                  /* [T, H/2]  masked residual codes */
+  uint8_t* rsf;                 /* [T, H/16] */
+  int32_t* sel13;               /* [rac_nsel_13] ascending */
+  float* a13_gs_out;            /* float[1] */
+  void* h_bf16;                 /* bf16 [A, I], dispatch order */
+  uint8_t* hq;                  /* [A, I/2] */
+  uint8_t* hsf;                 /* [A, I/16] linear */
+  uint8_t* r2q;                 /* [A, I/2] masked residual codes of h */
+  uint8_t* r2sf;                /* [A, I/16] */
+  int32_t* sel2;                /* [rac_nsel_2] ascending */
+  void* workspace;
+  size_t workspace_bytes;       /* >= quads_moe_workspace_bytes(T, H, I, E, topk, N) */
+} quads_moe_args;
+
+quads_status quads_moe_w4a4_rac(const quads_moe_args* args /* host */, void* cuda_stream);
+size_t quads_moe_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk,
+                                 int32_t N);
+/* Reads (with a device-to-host copy and a stream synchronise) the status word
+   that device-side bounded waits write into the workspace of an earlier
+   quads_moe_w4a4_rac call: QUADS_OK or QUADS_ERR_TIMEOUT. */
+quads_status quads_moe_async_status(const void* workspace, void* cuda_stream);
+
+/* Number of kernels the last quads_* call on this host thread enqueued. */
+int32_t quads_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QUADS_H_ */

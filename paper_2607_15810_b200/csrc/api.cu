@@ -1,0 +1,438 @@
+// C ABI entry points: argument checks, workspace carving, TMA descriptors and
+// the launch sequence of each public call.
+#include <mutex>
+
+#include "kernels.cuh"
+
+namespace quads {
+
+thread_local int g_launch_count = 0;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct DeviceInfo {
+  int sm_count = 0;
+  int cc_major = 0;
+  bool ok = false;
+};
+
+quads_status device_info(DeviceInfo* out) {
+  static std::mutex mu;
+  static DeviceInfo cache[64];
+  int dev = 0;
+  QUADS_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QUADS_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cache[dev].ok) {
+    QUADS_CUDA_OK(cudaDeviceGetAttribute(&cache[dev].sm_count, cudaDevAttrMultiProcessorCount, dev));
+    QUADS_CUDA_OK(cudaDeviceGetAttribute(&cache[dev].cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+    cache[dev].ok = true;
+  }
+  *out = cache[dev];
+  return cache[dev].cc_major == 10 ? QUADS_OK : QUADS_ERR_ARCH;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  });
+  return fn;
+}
+
+// 2D map over packed FP4 codes viewed as bytes: [rows, row_bytes], box 128 bytes x
+// 128 rows, 128-byte swizzle, zero fill outside.
+quads_status make_codes_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return QUADS_ERR_CUDA;
+  if (rows == 0) rows = 1;
+  cuuint64_t dims[2] = {row_bytes, rows};
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {128, 128};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? QUADS_OK : QUADS_ERR_CUDA;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// ------------------------------------------------------------------ workspace
+struct MoeLayout {
+  size_t header, amax, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
+  size_t perm, pos_pad, row_token, row_weight;
+  size_t partials13, scores13, sel13, mask13, xq_pad, xsf, rq_pad, rsf;
+  size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, out32;
+  size_t total;
+  int n_chunks, m_tiles_max, stats_ctas, rows_per_cta;
+};
+
+MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
+  MoeLayout L{};
+  const bool dense = (I == 0);
+  const int64_t A = dense ? T : (int64_t)T * topk;
+  const int Ee = dense ? 1 : E;
+  L.n_chunks = (T + kRouteTokensPerCta - 1) / kRouteTokensPerCta;
+  L.m_tiles_max = (int)(A / 128) + Ee;
+  L.stats_ctas = T < 592 * 4 ? (T + 3) / 4 : 592;
+  if (L.stats_ctas < 1) L.stats_ctas = 1;
+  L.rows_per_cta = (T + L.stats_ctas - 1) / L.stats_ctas;
+  if (L.rows_per_cta < 1) L.rows_per_cta = 1;
+  L.stats_ctas = (T + L.rows_per_cta - 1) / L.rows_per_cta;
+  if (L.stats_ctas < 1) L.stats_ctas = 1;
+  const size_t pad_rows = (size_t)L.m_tiles_max * 128;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+  L.header = take(kHdrWords * 4);
+  L.amax = take(16);
+  L.ids = take((size_t)A * 4);
+  L.wts = take((size_t)A * 4);
+  L.chunk_counts = take((size_t)L.n_chunks * Ee * 4);
+  L.chunk_base = take((size_t)L.n_chunks * Ee * 4);
+  L.offsets = take((size_t)(Ee + 1) * 4);
+  L.tile_prefix = take((size_t)(Ee + 1) * 4);
+  L.tile_expert = take((size_t)L.m_tiles_max * 4);
+  L.tile_rows = take((size_t)L.m_tiles_max * 4);
+  L.perm = take((size_t)A * 4);
+  L.pos_pad = take((size_t)A * 4);
+  L.row_token = take(pad_rows * 4);
+  L.row_weight = take(pad_rows * 4);
+  L.partials13 = take((size_t)L.stats_ctas * H * 4);
+  L.scores13 = take((size_t)H * 8);
+  L.sel13 = take((size_t)H * 4);
+  L.mask13 = take((size_t)H);
+  L.xq_pad = take(pad_rows * (H / 2));
+  L.xsf = take((size_t)L.m_tiles_max * (H / 64) * 512);
+  L.rq_pad = take(pad_rows * (H / 2));
+  L.rsf = take((size_t)L.m_tiles_max * (H / 64) * 512);
+  if (!dense) {
+    L.hq_pad = take(pad_rows * (I / 2));
+    L.hsf = take((size_t)L.m_tiles_max * (I / 64) * 512);
+    L.r2q_pad = take(pad_rows * (I / 2));
+    L.r2sf = take((size_t)L.m_tiles_max * (I / 64) * 512);
+    L.partials2 = take((size_t)L.m_tiles_max * 4 * I * 4);
+    L.scores2 = take((size_t)I * 8);
+    L.sel2 = take((size_t)I * 4);
+    L.mask2 = take((size_t)I);
+    L.out32 = take((size_t)T * H * 4);
+  }
+  (void)N;
+  L.total = o;
+  return L;
+}
+
+int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+
+quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
+                        int n_sel,
+                        double* scores, int32_t* sel_list, uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
+  score_reduce_kernel<<<(C + 31) / 32, 256, 0, st>>>(partials, n_part_ptr, n_part_mul, n_part_fixed, C, scores);
+  note_launch();
+  const int n2 = pow2_at_least(C);
+  const size_t smem = (size_t)n2 * 12 + (size_t)(C + 1) * 4;
+  static bool attr = false;
+  if (!attr) {
+    QUADS_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    attr = true;
+  }
+  select_kernel<<<1, 1024, smem, st>>>(scores, C, n_sel, n2, sel_list, mask, sel_export);
+  note_launch();
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
+}  // namespace
+}  // namespace quads
+
+using namespace quads;
+
+extern "C" {
+
+const char* quads_status_string(quads_status s) {
+  switch (s) {
+    case QUADS_OK: return "QUADS_OK";
+    case QUADS_ERR_NULL: return "QUADS_ERR_NULL: a required pointer is NULL";
+    case QUADS_ERR_SHAPE: return "QUADS_ERR_SHAPE: a size breaks a divisibility or range rule";
+    case QUADS_ERR_WORKSPACE: return "QUADS_ERR_WORKSPACE: workspace missing, misaligned or too small";
+    case QUADS_ERR_ARCH: return "QUADS_ERR_ARCH: the current device is not sm_100";
+    case QUADS_ERR_CUDA: return "QUADS_ERR_CUDA: a CUDA runtime or driver call failed";
+    case QUADS_ERR_TIMEOUT: return "QUADS_ERR_TIMEOUT: a bounded device-side wait gave up";
+    default: return "QUADS: unknown status";
+  }
+}
+
+size_t quads_sf_tiled_bytes(int64_t rows, int64_t K) {
+  if (rows < 0 || K < 0) return 0;
+  return (size_t)((rows + 127) / 128) * (size_t)((K + 63) / 64) * 512u;
+}
+
+size_t quads_quantize_workspace_bytes(void) { return 256; }
+size_t quads_fake_quant_workspace_bytes(int64_t n_tensors) {
+  return align_up((size_t)(n_tensors > 0 ? n_tensors : 1) * 4, 256);
+}
+int32_t quads_last_launch_count(void) { return g_launch_count; }
+
+static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t rows, int64_t K, int64_t ld,
+                                    int64_t tensor_stride, const float* gs_in, void* fq, uint8_t* q, uint8_t* sf,
+                                    float* gs_out, int sf_layout, void* workspace, size_t workspace_bytes,
+                                    cudaStream_t st) {
+  g_launch_count = 0;
+  if (rows < 0 || n_tensors < 0 || K <= 0 || (K % 16) != 0 || ld < K || (ld % 16) != 0) return QUADS_ERR_SHAPE;
+  if (sf_layout != QUADS_SF_LINEAR && sf_layout != QUADS_SF_TILED) return QUADS_ERR_SHAPE;
+  if (rows * (K / 16) > (int64_t)0x7FFFFFFF * 256 || n_tensors > 65535) return QUADS_ERR_SHAPE;
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < quads_fake_quant_workspace_bytes(n_tensors))
+    return QUADS_ERR_WORKSPACE;
+  if (n_tensors > 0 && rows > 0 && !x) return QUADS_ERR_NULL;
+  if (!aligned(x, 32) || !aligned(q, 8) || !aligned(fq, 32) || !aligned(sf, 4)) return QUADS_ERR_SHAPE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  if (n_tensors == 0) return QUADS_OK;
+  uint32_t* amax_bits = static_cast<uint32_t*>(workspace);
+  if (!gs_in) {
+    QUADS_CUDA_OK(cudaMemsetAsync(amax_bits, 0, (size_t)n_tensors * 4, st));
+    if (rows > 0) {
+      const int64_t chunks = rows * (K / 8);
+      int gx = (int)((chunks + 256 * 8 - 1) / (256 * 8));
+      const int cap = (di.sm_count * 8 + (int)n_tensors - 1) / (int)n_tensors;
+      if (gx > cap) gx = cap;
+      if (gx < 1) gx = 1;
+      amax_kernel<<<dim3(gx, (unsigned)n_tensors), 256, 0, st>>>(static_cast<const uint16_t*>(x), rows, K, ld,
+                                                                   tensor_stride, amax_bits);
+      note_launch();
+    }
+  }
+  const int64_t nblk = rows * (K / 16);
+  const unsigned gx = (unsigned)((nblk + 255) / 256);
+  const int64_t sf_stride = sf_layout == QUADS_SF_TILED ? (int64_t)quads_sf_tiled_bytes(rows, K) : rows * (K / 16);
+  quantize_kernel<<<dim3(gx > 0 ? gx : 1, (unsigned)n_tensors), 256, 0, st>>>(
+      static_cast<const uint16_t*>(x), rows, K, ld, tensor_stride, gs_in, amax_bits, q, sf,
+      static_cast<uint16_t*>(fq), gs_out, sf_layout == QUADS_SF_TILED, sf_stride);
+  note_launch();
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
+quads_status quads_quantize_nvfp4(const void* x, int64_t rows, int64_t K, int64_t ld, const float* gs_in,
+                                  uint8_t* q, uint8_t* sf, float* gs_out, int sf_layout, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+  if (rows > 0 && (!q || !sf)) return QUADS_ERR_NULL;
+  return quantize_common(x, 1, rows, K, ld, 0, gs_in, nullptr, q, sf, gs_out, sf_layout, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t N, int64_t K, void* w_fq,
+                                      uint8_t* q, uint8_t* sf, float* gs, int sf_layout, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream) {
+  if (!gs && n_tensors > 0) return QUADS_ERR_NULL;
+  return quantize_common(w, n_tensors, N, K, K, N * K, nullptr, w_fq, q, sf, gs, sf_layout, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t quads_moe_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk, int32_t N) {
+  if (T < 0 || H <= 0 || I < 0 || E < 1 || topk < 1) return 0;
+  return moe_layout(T, H, I, E, topk, N).total;
+}
+
+quads_status quads_moe_async_status(const void* workspace, void* cuda_stream) {
+  if (!workspace) return QUADS_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t v = 0;
+  QUADS_CUDA_OK(cudaMemcpyAsync(&v, static_cast<const int32_t*>(workspace) + kHdrStatus, 4, cudaMemcpyDeviceToHost, st));
+  QUADS_CUDA_OK(cudaStreamSynchronize(st));
+  return v == 0 ? QUADS_OK : (quads_status)v;
+}
+
+quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
+  g_launch_count = 0;
+  if (!a) return QUADS_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool dense = (a->I == 0);
+  const int T = a->T, H = a->H, I = a->I;
+  const int E = dense ? 1 : a->E, topk = dense ? 1 : a->topk;
+  const int N1 = dense ? a->N : 2 * I;            // weight rows of the first projection
+  if (T < 0 || H <= 0 || (H % 128) != 0 || I < 0 || (I % 128) != 0) return QUADS_ERR_SHAPE;
+  if (dense && (a->N <= 0 || (a->N % 128) != 0)) return QUADS_ERR_SHAPE;
+  if (!dense && (E < 1 || E > kMaxExperts || topk < 1 || topk > kMaxTopk || topk > E)) return QUADS_ERR_SHAPE;
+  if (a->rac_nsel_13 < 0 || a->rac_nsel_13 > H || (!dense && (a->rac_nsel_2 < 0 || a->rac_nsel_2 > I)))
+    return QUADS_ERR_SHAPE;
+  if ((int64_t)T * topk > 0x3FFFFFFF) return QUADS_ERR_SHAPE;
+  if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) return QUADS_ERR_NULL;
+  if (!dense && (!a->router_logits || !a->w2_q || !a->w2_sf || !a->w2_gs || !a->a2_gs)) return QUADS_ERR_NULL;
+  if (!aligned(a->x, 32) || !aligned(a->w13_q, 16) || !aligned(a->w13_sf, 16) || !aligned(a->out, 16) ||
+      (!dense && (!aligned(a->w2_q, 16) || !aligned(a->w2_sf, 16))))
+    return QUADS_ERR_SHAPE;
+  const MoeLayout L = moe_layout(T, H, I, E, topk, a->N);
+  if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < L.total) return QUADS_ERR_WORKSPACE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  if (T == 0) return QUADS_OK;
+
+  uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+  auto P = [&](size_t off) { return ws + off; };
+  int32_t* header = reinterpret_cast<int32_t*>(P(L.header));
+  uint32_t* amax_bits = reinterpret_cast<uint32_t*>(P(L.amax));
+  int32_t* ids = reinterpret_cast<int32_t*>(P(L.ids));
+  float* wts = reinterpret_cast<float*>(P(L.wts));
+  int32_t* offsets = reinterpret_cast<int32_t*>(P(L.offsets));
+  int32_t* tile_prefix = reinterpret_cast<int32_t*>(P(L.tile_prefix));
+  int32_t* tile_expert = reinterpret_cast<int32_t*>(P(L.tile_expert));
+  int32_t* tile_rows = reinterpret_cast<int32_t*>(P(L.tile_rows));
+  int32_t* perm = reinterpret_cast<int32_t*>(P(L.perm));
+  int32_t* pos_pad = reinterpret_cast<int32_t*>(P(L.pos_pad));
+  int32_t* row_token = reinterpret_cast<int32_t*>(P(L.row_token));
+  float* row_weight = reinterpret_cast<float*>(P(L.row_weight));
+  const uint16_t* x = static_cast<const uint16_t*>(a->x);
+  const int A = T * topk;
+  const size_t pad_rows = (size_t)L.m_tiles_max * 128;
+
+  // header (status word included) and the amax word start at zero
+  QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, L.ids, st));
+
+  // ---- per-tensor scale of x
+  if (!a->a13_gs) {
+    const int64_t chunks = (int64_t)T * (H / 8);
+    int gx = (int)((chunks + 2047) / 2048);
+    if (gx > di.sm_count * 8) gx = di.sm_count * 8;
+    amax_kernel<<<dim3(gx, 1), 256, 0, st>>>(x, T, H, H, 0, amax_bits);
+    note_launch();
+  }
+
+  // ---- routing and dispatch order
+  if (dense) {
+    dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, pos_pad, row_token, row_weight, tile_expert,
+                                                           tile_rows, header);
+    note_launch();
+  } else {
+    int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
+    int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
+    route_kernel<<<L.n_chunks, 256, 0, st>>>(a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts,
+                                              a->topk_ids, a->topk_w);
+    note_launch();
+    scan_kernel<<<1, 256, 0, st>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
+                                   tile_rows, header, a->expert_offsets);
+    note_launch();
+    permute_kernel<<<L.n_chunks, 256, 0, st>>>(T, E, topk, ids, wts, chunk_base, offsets, tile_prefix, perm,
+                                               pos_pad, row_token, row_weight, a->perm);
+    note_launch();
+  }
+
+  // ---- site 13: statistics, selection, quantize + residual + dispatch scatter
+  const int nsel13 = a->rac_nsel_13;
+  float* gs13_store = a->a13_gs_out;
+  uint8_t* mask13 = P(L.mask13);
+  if (nsel13 > 0 || a->xq || a->xsf || gs13_store) {
+    rac_stats_kernel<<<L.stats_ctas, H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32, 0, st>>>(
+        x, T, H, a->a13_gs, amax_bits, gs13_store, L.rows_per_cta, reinterpret_cast<float*>(P(L.partials13)),
+        a->xq, a->xsf);
+    note_launch();
+  }
+  if (nsel13 > 0) {
+    s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
+                   reinterpret_cast<double*>(P(L.scores13)), reinterpret_cast<int32_t*>(P(L.sel13)), mask13,
+                   a->sel13, st);
+    if (s != QUADS_OK) return s;
+  }
+  // the dispatch kernel needs the scale as a value in memory: the amax word or the caller's
+  {
+    const int64_t groups = (int64_t)T * (H / 64);
+    rac_dispatch_kernel<<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(
+        x, T, H, a->a13_gs, amax_bits, nsel13, mask13, topk, pos_pad, P(L.xq_pad), P(L.xsf), P(L.rq_pad),
+        P(L.rsf), a->rq, a->rsf);
+    note_launch();
+  }
+
+  // ---- tensor maps
+  CUtensorMap tm_x, tm_r, tm_w13;
+  if ((s = make_codes_map(&tm_x, P(L.xq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&tm_r, P(L.rq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&tm_w13, a->w13_q, (uint64_t)E * N1, H / 2)) != QUADS_OK) return s;
+
+  GemmParams g{};
+  g.K = H;
+  g.has_resid = nsel13 > 0;
+  g.header = header; g.tile_expert = tile_expert; g.tile_rows = tile_rows;
+  g.a_sf = P(L.xsf); g.r_sf = P(L.rsf);
+  g.b_sf = a->w13_sf; g.b_sf_expert_stride = quads_sf_tiled_bytes(N1, H);
+  g.b_gs = a->w13_gs; g.a_gs = a->a13_gs; g.a_amax_bits = amax_bits;
+  g.row_token = row_token; g.row_weight = row_weight;
+  g.tile_prefix = tile_prefix; g.offsets = offsets;
+  g.status = header + kHdrStatus;
+  g.b_rows_per_expert = N1;
+  if (dense) {
+    g.n_out = a->N;
+    g.n_tiles_n = (a->N + 255) / 256;
+    g.half1_row_offset = 128;
+    g.out_bf16 = static_cast<uint16_t*>(a->out);
+    return launch_gemm(kEpiStore, g, tm_x, tm_r, tm_w13, di.sm_count, st);
+  }
+  g.n_out = I;
+  g.n_tiles_n = I / 128;
+  g.half1_row_offset = I;
+  g.h_gs = a->a2_gs;
+  g.resid2 = a->rac_nsel_2 > 0 || a->r2q || a->r2sf;
+  g.hq_pad = P(L.hq_pad); g.hsf_tiled = P(L.hsf); g.r2q_pad = P(L.r2q_pad); g.r2sf_tiled = P(L.r2sf);
+  g.partials2 = reinterpret_cast<float*>(P(L.partials2));
+  g.h_export = static_cast<uint16_t*>(a->h_bf16);
+  if ((s = launch_gemm(kEpiSwiGLU, g, tm_x, tm_r, tm_w13, di.sm_count, st)) != QUADS_OK) return s;
+
+  // ---- site 2: selection and masking of the residual of h
+  const int nsel2 = a->rac_nsel_2;
+  uint8_t* mask2 = P(L.mask2);
+  if (nsel2 > 0) {
+    s = run_select(g.partials2, header + kHdrMTiles, 4 /* one partial row per tile and lane quadrant */, 0, I, nsel2,
+                   reinterpret_cast<double*>(P(L.scores2)), reinterpret_cast<int32_t*>(P(L.sel2)), mask2, a->sel2, st);
+    if (s != QUADS_OK) return s;
+    mask_codes_kernel<<<di.sm_count * 8, 256, 0, st>>>(P(L.r2q_pad), header + kHdrPaddedRows, I, mask2);
+    note_launch();
+  } else if (a->r2q) {
+    QUADS_CUDA_OK(cudaMemsetAsync(mask2, 0, I, st));
+  }
+  if (a->hq || a->hsf || a->r2q || a->r2sf) {
+    const int64_t n = (int64_t)A * (I / 16);
+    export_site2_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(A, I, perm, pos_pad, P(L.hq_pad), P(L.hsf),
+                                                                     P(L.r2q_pad), P(L.r2sf), mask2, a->hq, a->hsf,
+                                                                     a->r2q, a->r2sf);
+    note_launch();
+  }
+
+  // ---- second projection + weighted combine
+  float* out32 = reinterpret_cast<float*>(P(L.out32));
+  QUADS_CUDA_OK(cudaMemsetAsync(out32, 0, (size_t)T * H * 4, st));
+  CUtensorMap tm_h, tm_r2, tm_w2;
+  if ((s = make_codes_map(&tm_h, P(L.hq_pad), pad_rows, I / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&tm_r2, P(L.r2q_pad), pad_rows, I / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&tm_w2, a->w2_q, (uint64_t)E * H, I / 2)) != QUADS_OK) return s;
+  GemmParams g2 = g;
+  g2.K = I;
+  g2.has_resid = nsel2 > 0;
+  g2.a_sf = P(L.hsf); g2.r_sf = P(L.r2sf);
+  g2.b_sf = a->w2_sf; g2.b_sf_expert_stride = quads_sf_tiled_bytes(H, I);
+  g2.b_gs = a->w2_gs; g2.a_gs = a->a2_gs; g2.a_amax_bits = nullptr;
+  g2.b_rows_per_expert = H;
+  g2.n_out = H;
+  g2.n_tiles_n = (H + 255) / 256;
+  g2.half1_row_offset = 128;
+  g2.out_f32 = out32;
+  if ((s = launch_gemm(kEpiCombine, g2, tm_h, tm_r2, tm_w2, di.sm_count, st)) != QUADS_OK) return s;
+  const int64_t n4 = (int64_t)T * H / 4;
+  finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(out32, static_cast<uint16_t*>(a->out), n4);
+  note_launch();
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
+}  // extern "C"

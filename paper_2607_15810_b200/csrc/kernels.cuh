@@ -1,0 +1,93 @@
+// Kernel declarations shared by the translation units of libquads.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace quads {
+
+constexpr int kRouteTokensPerCta = 64;
+constexpr int kMaxTopk = 16;
+constexpr int kMaxExperts = 256;
+
+// header words written by the scan (device side sizes of the dispatch)
+enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, kHdrWords = 8 };
+
+// ---- quantize.cu
+__global__ void amax_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
+                            uint32_t* amax_bits);
+__global__ void quantize_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
+                                const float* gs_in, const uint32_t* amax_bits, uint8_t* q, uint8_t* sf,
+                                uint16_t* fq, float* gs_out, int sf_tiled, int64_t sf_tensor_stride);
+__global__ void rac_stats_kernel(const uint16_t* x, int T, int H, const float* gs_in, const uint32_t* amax_bits,
+                                 float* gs_store, int rows_per_cta, float* partials, uint8_t* xq_out,
+                                 uint8_t* xsf_out);
+__global__ void score_reduce_kernel(const float* partials, const int* n_part_ptr, int n_part_mul,
+                                    int n_part_fixed, int C, double* scores);
+__global__ void select_kernel(const double* scores, int C, int n_sel, int n_pow2, int32_t* sel_list,
+                              uint8_t* mask, int32_t* sel_export);
+__global__ void rac_dispatch_kernel(const uint16_t* x, int T, int H, const float* gs_in,
+                                    const uint32_t* amax_bits, int n_sel,
+                                    const uint8_t* mask, int topk, const int32_t* pos_pad, uint8_t* xq_pad,
+                                    uint8_t* xsf_tiled, uint8_t* rq_pad, uint8_t* rsf_tiled, uint8_t* rq_out,
+                                    uint8_t* rsf_out);
+__global__ void mask_codes_kernel(uint8_t* codes, const int* n_rows_ptr, int C, const uint8_t* mask);
+__global__ void finalize_kernel(const float* acc, uint16_t* out, int64_t n4);
+__global__ void export_site2_kernel(int A, int I, const int32_t* perm, const int32_t* pos_pad,
+                                    const uint8_t* hq_pad, const uint8_t* hsf_tiled, const uint8_t* r2q_pad,
+                                    const uint8_t* r2sf_tiled, const uint8_t* mask2, uint8_t* hq, uint8_t* hsf,
+                                    uint8_t* r2q, uint8_t* r2sf);
+
+// ---- routing.cu
+__global__ void route_kernel(const float* logits, int T, int E, int topk, int renormalize, int32_t* ids,
+                             float* wts, int32_t* chunk_counts, int32_t* ids_out, float* wts_out);
+__global__ void scan_kernel(int E, int n_chunks, const int32_t* chunk_counts, int32_t* chunk_base,
+                            int32_t* offsets, int32_t* tile_prefix, int32_t* tile_expert, int32_t* tile_rows,
+                            int32_t* header, int32_t* offsets_out);
+__global__ void permute_kernel(int T, int E, int topk, const int32_t* ids, const float* wts,
+                               const int32_t* chunk_base, const int32_t* offsets, const int32_t* tile_prefix,
+                               int32_t* perm, int32_t* pos_pad, int32_t* row_token, float* row_weight,
+                               int32_t* perm_out);
+__global__ void dense_dispatch_kernel(int T, int32_t* pos_pad, int32_t* row_token, float* row_weight,
+                                      int32_t* tile_expert, int32_t* tile_rows, int32_t* header);
+
+// ---- gemm.cu
+enum { kEpiStore = 0, kEpiSwiGLU = 1, kEpiCombine = 2 };
+
+struct GemmParams {
+  int K;                 // contraction length in elements (multiple of 64)
+  int n_tiles_n;         // tiles along the output-feature dimension
+  int n_out;             // output features (I for SwiGLU, else N)
+  int b_rows_per_expert; // weight rows per expert
+  int half1_row_offset;  // weight-row distance from the tile's first half to its second half
+  int has_resid;         // 1: also accumulate the (negated, masked) residual operand
+  const int32_t* header;
+  const int32_t* tile_expert;
+  const int32_t* tile_rows;
+  const uint8_t* a_sf;   // tiled scales of the main activation operand (padded dispatch rows)
+  const uint8_t* r_sf;   // tiled scales of the residual operand
+  const uint8_t* b_sf;   // tiled weight scales, one block per expert
+  size_t b_sf_expert_stride;
+  const float* b_gs;     // [E] per-tensor weight scales
+  const float* a_gs;     // per-tensor activation scale (pointer), or NULL ...
+  const uint32_t* a_amax_bits;  // ... then derived from this amax word
+  // epilogue: store / combine
+  const int32_t* row_token;
+  const float* row_weight;
+  uint16_t* out_bf16;    // kEpiStore: [T, n_out]
+  float* out_f32;        // kEpiCombine: [T, n_out] accumulation buffer
+  // epilogue: SwiGLU + requantize (site 2)
+  const float* h_gs;     // per-tensor scale of h
+  int resid2;            // 1: also emit the residual of h and its column statistics
+  uint8_t* hq_pad; uint8_t* hsf_tiled; uint8_t* r2q_pad; uint8_t* r2sf_tiled;
+  float* partials2;      // [4 * m_tiles, n_out]
+  uint16_t* h_export;    // optional bf16 [A, n_out] in dispatch order
+  const int32_t* tile_prefix;
+  const int32_t* offsets;
+  int32_t* status;       // device status word (QUADS_ERR_TIMEOUT on a failed wait)
+};
+
+quads_status launch_gemm(int epi, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
+                         const CUtensorMap& tm_b, int n_sms, cudaStream_t stream);
+
+}  // namespace quads

@@ -1,0 +1,374 @@
+// Streaming kernels: tensor amax, NVFP4 quantize / fake-quant, RAC statistics,
+// channel selection, masked residual quantize + dispatch scatter, small fix-ups.
+// All HBM- or latency-bound; no tensor cores here.
+#include "kernels.cuh"
+
+namespace quads {
+
+// ---------------------------------------------------------------------------
+// amax over bf16 tensors.  gridDim.y = tensor; magnitudes compared as 15-bit
+// integers (two per 32-bit word); result = bf16 bit pattern << 16 = float bits.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) amax_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K,
+                                                   int64_t ld, int64_t tensor_stride,
+                                                   uint32_t* __restrict__ amax_bits) {
+  const uint16_t* base = x + (size_t)blockIdx.y * tensor_stride;
+  const int64_t k8 = K >> 3;
+  const int64_t chunks = rows * k8;
+  uint32_t m = 0;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  if (ld == K) {
+    const uint4* p = reinterpret_cast<const uint4*>(base);
+    int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; c + 3 * stride < chunks; c += 4 * stride) {
+      uint4 v0 = __ldg(p + c), v1 = __ldg(p + c + stride), v2 = __ldg(p + c + 2 * stride),
+            v3 = __ldg(p + c + 3 * stride);
+      uint32_t a = __vmaxu2(__vmaxu2(v0.x & 0x7FFF7FFFu, v0.y & 0x7FFF7FFFu),
+                            __vmaxu2(v0.z & 0x7FFF7FFFu, v0.w & 0x7FFF7FFFu));
+      uint32_t b = __vmaxu2(__vmaxu2(v1.x & 0x7FFF7FFFu, v1.y & 0x7FFF7FFFu),
+                            __vmaxu2(v1.z & 0x7FFF7FFFu, v1.w & 0x7FFF7FFFu));
+      uint32_t c2 = __vmaxu2(__vmaxu2(v2.x & 0x7FFF7FFFu, v2.y & 0x7FFF7FFFu),
+                             __vmaxu2(v2.z & 0x7FFF7FFFu, v2.w & 0x7FFF7FFFu));
+      uint32_t d = __vmaxu2(__vmaxu2(v3.x & 0x7FFF7FFFu, v3.y & 0x7FFF7FFFu),
+                            __vmaxu2(v3.z & 0x7FFF7FFFu, v3.w & 0x7FFF7FFFu));
+      m = __vmaxu2(m, __vmaxu2(__vmaxu2(a, b), __vmaxu2(c2, d)));
+    }
+    for (; c < chunks; c += stride) {
+      uint4 v = __ldg(p + c);
+      m = __vmaxu2(m, __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu),
+                               __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)));
+    }
+  } else {
+    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < chunks; c += stride) {
+      const int64_t r = c / k8, cc = c - r * k8;
+      uint4 v = __ldg(reinterpret_cast<const uint4*>(base + r * ld + cc * 8));
+      m = __vmaxu2(m, __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu),
+                               __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu)));
+    }
+  }
+  uint32_t s = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s = max(s, __shfl_xor_sync(0xFFFFFFFFu, s, o));
+  __shared__ uint32_t wmax[8];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t t = 0;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t = max(t, wmax[i]);
+    if (t) atomicMax(amax_bits + blockIdx.y, t << 16);
+  }
+}
+
+__device__ __forceinline__ float gs_from_amax_bits(uint32_t bits) {
+  const float amax = __uint_as_float(bits);
+  return amax > 0.f ? __fdiv_rn(amax, kGlobalDiv) : 1.0f;
+}
+
+// ---------------------------------------------------------------------------
+// NVFP4 quantize / fake-quant: one thread per 16-element block.
+// gridDim.y = tensor.  The per-tensor scale comes from gs_in[tensor] when
+// gs_in != NULL, else from amax_bits[tensor].
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
+                const float* __restrict__ gs_in, const uint32_t* __restrict__ amax_bits,
+                uint8_t* __restrict__ q, uint8_t* __restrict__ sf, uint16_t* __restrict__ fq,
+                float* __restrict__ gs_out, int sf_tiled, int64_t sf_tensor_stride) {
+  const int t = blockIdx.y;
+  const float gs = gs_in ? gs_in[t] : gs_from_amax_bits(amax_bits[t]);
+  if (gs_out && blockIdx.x == 0 && threadIdx.x == 0) gs_out[t] = gs;
+  const int64_t k16 = K >> 4;
+  const int64_t nblk = rows * k16;
+  const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= nblk) return;
+  const int64_t r = b / k16, kb = b - r * k16;
+  const uint16_t* src = x + (size_t)t * tensor_stride + r * ld + kb * 16;
+  uint4 v0, v1;
+  ldg256(src, v0, v1);
+  float f[16];
+  unpack8(v0, f);
+  unpack8(v1, f + 8);
+  const BlockQ bq = quantize_block(f, gs);
+  const size_t row_global = (size_t)t * rows + r;
+  if (q) *reinterpret_cast<uint2*>(q + row_global * (K >> 1) + kb * 8) = make_uint2(bq.lo, bq.hi);
+  if (sf) {
+    uint8_t* sft = sf + (size_t)t * sf_tensor_stride;
+    if (sf_tiled) sft[sf_tiled_offset(r, kb, (K + 63) >> 6)] = (uint8_t)bq.sf8;
+    else sft[r * k16 + kb] = (uint8_t)bq.sf8;
+  }
+  if (fq) {
+    float o[16];
+    dequant_block(bq, o);
+    uint4 w0, w1;
+    w0.x = f32x2_to_bf16x2(o[0], o[1]);   w0.y = f32x2_to_bf16x2(o[2], o[3]);
+    w0.z = f32x2_to_bf16x2(o[4], o[5]);   w0.w = f32x2_to_bf16x2(o[6], o[7]);
+    w1.x = f32x2_to_bf16x2(o[8], o[9]);   w1.y = f32x2_to_bf16x2(o[10], o[11]);
+    w1.z = f32x2_to_bf16x2(o[12], o[13]); w1.w = f32x2_to_bf16x2(o[14], o[15]);
+    uint4* dst = reinterpret_cast<uint4*>(fq + (size_t)t * rows * K + r * K + kb * 16);
+    dst[0] = w0;
+    dst[1] = w1;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// RAC statistics at an activation site (Eq. channel-score): per-channel sum of
+// squared residuals of Q_A(x) over the rows this CTA owns, written as one
+// partial row per CTA (reduced later in a fixed order).  Optionally exports the
+// codes / scales of Q_A(x) in token order.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+rac_stats_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __restrict__ gs_in,
+                 const uint32_t* __restrict__ amax_bits, float* __restrict__ gs_store,
+                 int rows_per_cta, float* __restrict__ partials, uint8_t* __restrict__ xq_out,
+                 uint8_t* __restrict__ xsf_out) {
+  const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
+  if (gs_store && blockIdx.x == 0 && threadIdx.x == 0) gs_store[0] = gs;
+  const int k16 = H >> 4;
+  const int r0 = blockIdx.x * rows_per_cta;
+  const int r1 = min(T, r0 + rows_per_cta);
+  for (int kb = threadIdx.x; kb < k16; kb += blockDim.x) {
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    for (int r = r0; r < r1; ++r) {
+      uint4 v0, v1;
+      ldg256(x + (size_t)r * H + kb * 16, v0, v1);
+      float f[16], o[16];
+      unpack8(v0, f);
+      unpack8(v1, f + 8);
+      const BlockQ bq = quantize_block(f, gs);
+      dequant_block(bq, o);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float d = __fsub_rn(o[i], f[i]);
+        acc[i] = __fmaf_rn(d, d, acc[i]);
+      }
+      if (xq_out) *reinterpret_cast<uint2*>(xq_out + (size_t)r * (H >> 1) + kb * 8) = make_uint2(bq.lo, bq.hi);
+      if (xsf_out) xsf_out[(size_t)r * k16 + kb] = (uint8_t)bq.sf8;
+    }
+    float4* dst = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * H + kb * 16);
+    dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    dst[2] = make_float4(acc[8], acc[9], acc[10], acc[11]);
+    dst[3] = make_float4(acc[12], acc[13], acc[14], acc[15]);
+  }
+}
+
+// Sum `n_part` partial rows of width C into float64 scores, fixed order.
+// grid = C/32 CTAs of 256 threads: 32 columns x 8 interleaved slices.
+__global__ void __launch_bounds__(256)
+score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ n_part_ptr, int n_part_mul,
+                    int n_part_fixed, int C, double* __restrict__ scores) {
+  const int n_part = n_part_ptr ? *n_part_ptr * n_part_mul : n_part_fixed;
+  const int col = blockIdx.x * 32 + (threadIdx.x & 31);
+  const int slice = threadIdx.x >> 5;
+  double s = 0.0;
+  if (col < C)
+    for (int p = slice; p < n_part; p += 8) s += (double)partials[(size_t)p * C + col];
+  __shared__ double sm[8][32];
+  sm[slice][threadIdx.x & 31] = s;
+  __syncthreads();
+  if (slice == 0 && col < C) {
+    double t = 0.0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x & 31];
+    scores[col] = t;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Channel selection (Eq. channel-select): the n_sel largest scores, ties to the
+// lower index.  One CTA; bitonic sort of (score, index) in shared memory, then
+// the ascending index list and a byte mask.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+select_kernel(const double* __restrict__ scores, int C, int n_sel, int n_pow2, int32_t* __restrict__ sel_list,
+              uint8_t* __restrict__ mask, int32_t* __restrict__ sel_export) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* key = reinterpret_cast<double*>(smem_raw);
+  int* idx = reinterpret_cast<int*>(key + n_pow2);
+  int* flag = idx + n_pow2;          // [C + 1] prefix counts
+  const int tid = threadIdx.x, nt = blockDim.x;
+  for (int i = tid; i < n_pow2; i += nt) {
+    key[i] = i < C ? scores[i] : -1.0;
+    idx[i] = i;
+  }
+  __syncthreads();
+  // "a before b" when a has the larger score, or equal score and lower index
+  for (int k = 2; k <= n_pow2; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < n_pow2; i += nt) {
+        const int p = i ^ j;
+        if (p > i) {
+          const double ka = key[i], kb = key[p];
+          const int ia = idx[i], ib = idx[p];
+          const bool a_first = (ka > kb) || (ka == kb && ia < ib);
+          const bool up = ((i & k) == 0);
+          if (up ? !a_first : a_first) {
+            key[i] = kb; key[p] = ka;
+            idx[i] = ib; idx[p] = ia;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  for (int i = tid; i < C; i += nt) flag[i] = 0;
+  __syncthreads();
+  for (int i = tid; i < n_sel; i += nt) flag[idx[i]] = 1;
+  __syncthreads();
+  for (int i = tid; i < C; i += nt) mask[i] = (uint8_t)flag[i];
+  __syncthreads();
+  // ascending list: serial chunks per thread, then a scan of chunk totals
+  __shared__ int chunk_tot[1024];
+  const int per = (C + nt - 1) / nt;
+  const int c0 = tid * per, c1 = min(C, c0 + per);
+  int cnt = 0;
+  for (int i = c0; i < c1; ++i) cnt += flag[i];
+  chunk_tot[tid] = cnt;
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int i = 0; i < nt; ++i) { const int c = chunk_tot[i]; chunk_tot[i] = run; run += c; }
+  }
+  __syncthreads();
+  int pos = chunk_tot[tid];
+  for (int i = c0; i < c1; ++i)
+    if (flag[i]) {
+      sel_list[pos] = i;
+      if (sel_export) sel_export[pos] = i;
+      ++pos;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Site-13 dispatch: for token row t and a group of four scale blocks (64
+// channels) recompute Q_A(x), form the residual, quantize it with the same
+// per-tensor scale, clear unselected channels (Eq. residual-recon), and write
+// both into every dispatched copy of the row (padded dispatch order, tiled
+// scale layout).  Residual codes are stored NEGATED (sign bit flipped) so the
+// GEMM can accumulate W Q(x) + W (-M Q(dx)) with two plain MMAs.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t nibble_mask8(const uint8_t* m) {
+  // m[0..7] in {0,1} -> 0xF per selected nibble
+  const uint2 v = *reinterpret_cast<const uint2*>(m);
+  uint32_t out = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out |= ((v.x >> (8 * i)) & 1u) * (0xFu << (4 * i));
+    out |= ((v.y >> (8 * i)) & 1u) * (0xFu << (16 + 4 * i));
+  }
+  return out;
+}
+
+__global__ void __launch_bounds__(256)
+rac_dispatch_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __restrict__ gs_in,
+                    const uint32_t* __restrict__ amax_bits, int n_sel, const uint8_t* __restrict__ mask, int topk, const int32_t* __restrict__ pos_pad,
+                    uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled, uint8_t* __restrict__ rq_pad,
+                    uint8_t* __restrict__ rsf_tiled, uint8_t* __restrict__ rq_out, uint8_t* __restrict__ rsf_out) {
+  const int groups = H >> 6;
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= (int64_t)T * groups) return;
+  const int t = (int)(g / groups), kg = (int)(g - (int64_t)t * groups);
+  const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
+  uint32_t xc[8], rc[8], xs = 0, rs = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int kb = kg * 4 + j;
+    uint4 v0, v1;
+    ldg256(x + (size_t)t * H + kb * 16, v0, v1);
+    float f[16];
+    unpack8(v0, f);
+    unpack8(v1, f + 8);
+    const BlockQ bq = quantize_block(f, gs);
+    xc[2 * j] = bq.lo; xc[2 * j + 1] = bq.hi;
+    xs |= bq.sf8 << (8 * j);
+    if (n_sel > 0) {
+      float o[16];
+      dequant_block(bq, o);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) o[i] = __fsub_rn(o[i], f[i]);
+      const BlockQ br = quantize_block(o, gs);
+      const uint32_t mlo = nibble_mask8(mask + kb * 16), mhi = nibble_mask8(mask + kb * 16 + 8);
+      rc[2 * j] = br.lo & mlo; rc[2 * j + 1] = br.hi & mhi;
+      rs |= br.sf8 << (8 * j);
+    }
+  }
+  const int kt_count = H >> 6;
+  if (n_sel > 0 && rq_out) {
+    uint4* d = reinterpret_cast<uint4*>(rq_out + (size_t)t * (H >> 1) + kg * 32);
+    d[0] = make_uint4(rc[0], rc[1], rc[2], rc[3]);
+    d[1] = make_uint4(rc[4], rc[5], rc[6], rc[7]);
+    *reinterpret_cast<uint32_t*>(rsf_out + (size_t)t * (H >> 4) + kg * 4) = rs;
+  }
+  for (int s = 0; s < topk; ++s) {
+    const int p = pos_pad[t * topk + s];
+    uint4* d = reinterpret_cast<uint4*>(xq_pad + (size_t)p * (H >> 1) + kg * 32);
+    d[0] = make_uint4(xc[0], xc[1], xc[2], xc[3]);
+    d[1] = make_uint4(xc[4], xc[5], xc[6], xc[7]);
+    const size_t so = sf_tiled_offset(p, kg * 4, kt_count);
+    *reinterpret_cast<uint32_t*>(xsf_tiled + so) = xs;
+    if (n_sel > 0) {
+      uint4* e = reinterpret_cast<uint4*>(rq_pad + (size_t)p * (H >> 1) + kg * 32);
+      e[0] = make_uint4(rc[0] ^ 0x88888888u, rc[1] ^ 0x88888888u, rc[2] ^ 0x88888888u, rc[3] ^ 0x88888888u);
+      e[1] = make_uint4(rc[4] ^ 0x88888888u, rc[5] ^ 0x88888888u, rc[6] ^ 0x88888888u, rc[7] ^ 0x88888888u);
+      *reinterpret_cast<uint32_t*>(rsf_tiled + so) = rs;
+    }
+  }
+}
+
+// Clear (in place) the codes of unselected channels of a padded [rows, C/2]
+// code matrix; one thread per 16 bytes (32 channels).
+__global__ void __launch_bounds__(256)
+mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_ptr, int C,
+                  const uint8_t* __restrict__ mask) {
+  const int per_row = C >> 5;
+  const int64_t n = (int64_t)(*n_rows_ptr) * per_row;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % per_row);
+    uint4* p = reinterpret_cast<uint4*>(codes) + i;
+    uint4 v = *p;
+    const uint8_t* m = mask + c * 32;
+    v.x &= nibble_mask8(m); v.y &= nibble_mask8(m + 8);
+    v.z &= nibble_mask8(m + 16); v.w &= nibble_mask8(m + 24);
+    *p = v;
+  }
+}
+
+// out32 [n] float -> bf16
+__global__ void __launch_bounds__(256)
+finalize_kernel(const float* __restrict__ acc, uint16_t* __restrict__ out, int64_t n4) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 v = reinterpret_cast<const float4*>(acc)[i];
+  reinterpret_cast<uint2*>(out)[i] = make_uint2(f32x2_to_bf16x2(v.x, v.y), f32x2_to_bf16x2(v.z, v.w));
+}
+
+// Export of padded dispatch-order buffers into linear dispatch order.
+// One thread per (dispatched row, 16-channel block).
+__global__ void __launch_bounds__(256)
+export_site2_kernel(int A, int I, const int32_t* __restrict__ perm, const int32_t* __restrict__ pos_pad,
+                    const uint8_t* __restrict__ hq_pad, const uint8_t* __restrict__ hsf_tiled,
+                    const uint8_t* __restrict__ r2q_pad, const uint8_t* __restrict__ r2sf_tiled,
+                    const uint8_t* __restrict__ mask2, uint8_t* __restrict__ hq, uint8_t* __restrict__ hsf, uint8_t* __restrict__ r2q,
+                    uint8_t* __restrict__ r2sf) {
+  const int k16 = I >> 4;
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (int64_t)A * k16) return;
+  const int row = (int)(i / k16), kb = (int)(i - (int64_t)row * k16);
+  const int p = pos_pad[perm[row]];
+  const size_t so = sf_tiled_offset(p, kb, I >> 6);
+  if (hq) *reinterpret_cast<uint2*>(hq + (size_t)row * (I >> 1) + kb * 8) =
+      *reinterpret_cast<const uint2*>(hq_pad + (size_t)p * (I >> 1) + kb * 8);
+  if (hsf) hsf[(size_t)row * k16 + kb] = hsf_tiled[so];
+  if (r2q) {
+    uint2 v = *reinterpret_cast<const uint2*>(r2q_pad + (size_t)p * (I >> 1) + kb * 8);
+    // stored negated: flip the signs back, then clear the unselected channels again
+    v.x = (v.x ^ 0x88888888u) & nibble_mask8(mask2 + kb * 16);
+    v.y = (v.y ^ 0x88888888u) & nibble_mask8(mask2 + kb * 16 + 8);
+    *reinterpret_cast<uint2*>(r2q + (size_t)row * (I >> 1) + kb * 8) = v;
+  }
+  if (r2sf) r2sf[(size_t)row * k16 + kb] = r2sf_tiled[so];
+}
+
+}  // namespace quads

@@ -1,0 +1,168 @@
+// Top-k routing, per-expert histogram, exclusive scan and the stable dispatch
+// permutation.  Integer outputs are deterministic: assignments (token, slot)
+// end up sorted by (expert, token, slot).
+#include "kernels.cuh"
+
+namespace quads {
+
+// One warp per token.  E <= 256.  Top-k by logit, ties to the lower expert id,
+// slots in descending-logit order; weights = softmax over all experts at the
+// chosen ones, optionally renormalised.  Each CTA (kRouteTokensPerCta tokens)
+// also writes its per-expert assignment counts: chunk_counts[cta][E].
+__global__ void __launch_bounds__(256)
+route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
+             int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
+             int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
+  __shared__ int hist[256];
+  for (int i = threadIdx.x; i < E; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t0 = blockIdx.x * kRouteTokensPerCta;
+  for (int tt = warp; tt < kRouteTokensPerCta; tt += 8) {
+    const int t = t0 + tt;
+    if (t >= T) break;
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int e = j * 32 + lane;
+      v[j] = e < E ? logits[(size_t)t * E + e] : -INFINITY;
+    }
+    // softmax denominator over all experts
+    float mx = v[0];
+#pragma unroll
+    for (int j = 1; j < 8; ++j) mx = fmaxf(mx, v[j]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sum += (j * 32 + lane < E) ? expf(v[j] - mx) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    float my_w = 0.f;      // lane s keeps slot s
+    int my_id = -1;
+    float wsum = 0.f;
+    for (int s = 0; s < topk; ++s) {
+      float bv = -INFINITY;
+      int be = 0x7FFFFFFF;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int e = j * 32 + lane;
+        if (e < E && (v[j] > bv)) { bv = v[j]; be = e; }    // ascending e within a lane: first max wins
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+        const int oe = __shfl_xor_sync(0xFFFFFFFFu, be, o);
+        if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
+      }
+      const float w = expf(bv - mx) / sum;
+      wsum += w;
+      if (lane == s) { my_w = w; my_id = be; }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (j * 32 + lane == be) v[j] = -INFINITY;         // remove the winner
+    }
+    if (lane < topk) {
+      if (renormalize) my_w = my_w / wsum;
+      ids[(size_t)t * topk + lane] = my_id;
+      wts[(size_t)t * topk + lane] = my_w;
+      if (ids_out) ids_out[(size_t)t * topk + lane] = my_id;
+      if (wts_out) wts_out[(size_t)t * topk + lane] = my_w;
+      atomicAdd(&hist[my_id], 1);
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < E; i += blockDim.x) chunk_counts[(size_t)blockIdx.x * E + i] = hist[i];
+}
+
+// One CTA.  Per expert: exclusive prefix over chunks, total count; then the
+// exclusive scan over experts of counts (offsets) and of 128-row tile counts
+// (tile_prefix), the tile -> (expert, valid rows) map, and the header.
+__global__ void __launch_bounds__(256)
+scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32_t* __restrict__ chunk_base,
+            int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tile_expert,
+            int32_t* __restrict__ tile_rows, int32_t* __restrict__ header, int32_t* __restrict__ offsets_out) {
+  __shared__ int cnt[256];
+  __shared__ int off[257];
+  __shared__ int tpre[257];
+  const int e = threadIdx.x;
+  if (e < E) {
+    int run = 0;
+    for (int c = 0; c < n_chunks; ++c) {
+      const int v = chunk_counts[(size_t)c * E + e];
+      chunk_base[(size_t)c * E + e] = run;
+      run += v;
+    }
+    cnt[e] = run;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int a = 0, t = 0;
+    for (int i = 0; i < E; ++i) {
+      off[i] = a; tpre[i] = t;
+      a += cnt[i];
+      t += (cnt[i] + 127) >> 7;
+    }
+    off[E] = a; tpre[E] = t;
+    header[kHdrMTiles] = t;
+    header[kHdrPaddedRows] = t * 128;
+    header[kHdrAssignments] = a;
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i <= E; i += blockDim.x) {
+    offsets[i] = off[i];
+    tile_prefix[i] = tpre[i];
+    if (offsets_out) offsets_out[i] = off[i];
+  }
+  if (e < E) {
+    const int n_t = tpre[e + 1] - tpre[e];
+    for (int m = 0; m < n_t; ++m) {
+      tile_expert[tpre[e] + m] = e;
+      tile_rows[tpre[e] + m] = min(128, cnt[e] - m * 128);
+    }
+  }
+}
+
+// One CTA per routing chunk, one thread per expert: walk the chunk's
+// assignments in (token, slot) order and hand out consecutive rows.
+__global__ void __launch_bounds__(256)
+permute_kernel(int T, int E, int topk, const int32_t* __restrict__ ids, const float* __restrict__ wts,
+               const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ offsets,
+               const int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ pos_pad,
+               int32_t* __restrict__ row_token, float* __restrict__ row_weight, int32_t* __restrict__ perm_out) {
+  __shared__ int sid[kRouteTokensPerCta * kMaxTopk];
+  const int t0 = blockIdx.x * kRouteTokensPerCta;
+  const int n_tok = min(kRouteTokensPerCta, T - t0);
+  const int n = n_tok * topk;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) sid[i] = ids[(size_t)t0 * topk + i];
+  __syncthreads();
+  const int e = threadIdx.x;
+  if (e >= E) return;
+  int run = chunk_base[(size_t)blockIdx.x * E + e];
+  const int row0 = offsets[e], pad0 = tile_prefix[e] * 128;
+  for (int i = 0; i < n; ++i) {
+    if (sid[i] == e) {
+      const int flat = t0 * topk + i;
+      perm[row0 + run] = flat;
+      if (perm_out) perm_out[row0 + run] = flat;
+      const int p = pad0 + run;
+      pos_pad[flat] = p;
+      row_token[p] = flat / topk;
+      row_weight[p] = wts[flat];
+      ++run;
+    }
+  }
+}
+
+// Dense mode: identity dispatch of T rows to a single "expert".
+__global__ void __launch_bounds__(256)
+dense_dispatch_kernel(int T, int32_t* __restrict__ pos_pad, int32_t* __restrict__ row_token,
+                      float* __restrict__ row_weight, int32_t* __restrict__ tile_expert,
+                      int32_t* __restrict__ tile_rows, int32_t* __restrict__ header) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  const int m_tiles = (T + 127) >> 7;
+  if (i < T) { pos_pad[i] = i; row_token[i] = i; row_weight[i] = 1.f; }
+  if (i < m_tiles) { tile_expert[i] = 0; tile_rows[i] = min(128, T - i * 128); }
+  if (i == 0) { header[kHdrMTiles] = m_tiles; header[kHdrPaddedRows] = m_tiles * 128; header[kHdrAssignments] = T; }
+}
+
+}  // namespace quads

@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the NVFP4 W4A4+RAC MoE layer forward on B200.
+
+  python bench.py --gpus N --steps K --warmup W [--workload prefill|decode|large]
+                  [--variant both|w13|plain] [--impl reference]
+
+A step is one pass of the whole hot path (activation amax, routing + dispatch,
+RAC statistics / selection / residual quantize, both grouped GEMMs with their
+fused epilogues, combine) over one batch of seeded synthetic input.  Rank 0
+prints ONE JSON line.  With N > 1 (torchrun) every rank runs its own replica of
+the layer on its own batch (no data-path collective; weak scaling).
+`--impl reference` times the CPU oracle on a bounded sample of the same
+workload on the host cores."""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="prefill", choices=["prefill", "decode", "large"])
+    ap.add_argument("--variant", default="both", choices=["both", "w13", "plain"])
+    ap.add_argument("--no-aux", action="store_true", help="skip the auxiliary quantize / fake-quant / decode numbers")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def nsel_of(shape, variant):
+    n13 = 0 if variant == "plain" else shape.H // 2
+    n2 = shape.I // 2 if variant == "both" else 0
+    return n13, n2
+
+
+def workload_config(shape, variant, extra=None):
+    n13, n2 = nsel_of(shape, variant)
+    cfg = {"workload": "moe_%s_T%d_H%d_E%d_top%d_I%d" % (shape.name, shape.T, shape.H, shape.E, shape.topk, shape.I),
+           "variant": {"both": "RAC 50% at W13 and W2 inputs", "w13": "RAC 50% at W13 input only",
+                       "plain": "plain W4A4"}[variant],
+           "rac_nsel_13": n13, "rac_nsel_2": n2, "tokens": shape.T,
+           "skew": "experts 0..%d get %.0f%% of assignments" % (shape.hot_experts - 1, shape.hot_share * 100)
+           if shape.hot_experts else "none",
+           "l2": "256 MB buffer written between timed iterations"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ----------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(shape, variant, budget_s):
+    """Prepare a bounded sample of the workload for the CPU oracle: the first
+    T_s tokens of the batch (all dims of the layer unchanged).  Returns a
+    callable running one oracle step and the sample description."""
+    import numpy as np
+    import torch
+    from oracle import formats as F
+    from oracle import moe as M
+    from oracle import nvfp4 as Q
+    from paper_2607_15810_b200 import synth
+
+    n13, n2 = nsel_of(shape, variant)
+    # the oracle dequantizes each expert it meets (~0.15 s each at these sizes)
+    n_exp = max(8, min(shape.E, int(budget_s / 0.2)))
+    T_s = max(1, n_exp // shape.topk)
+    x, _ = synth.activations(shape)
+    lg = synth.router_logits(shape)
+    x = x[:T_s].to(torch.float32).numpy()
+    lg = lg[:T_s].numpy()
+    ids, _ = M.route(lg, shape.topk, True)
+    experts = sorted(set(int(e) for e in ids.reshape(-1)))
+    I, H, E = shape.I, shape.H, shape.E
+    w13 = dict(codes=np.zeros((E, 2 * I, H), np.uint8), sf=np.zeros((E, 2 * I, H // 16), np.uint8),
+               gs=np.ones(E, np.float32))
+    w2 = dict(codes=np.zeros((E, H, I), np.uint8), sf=np.zeros((E, H, I // 16), np.uint8), gs=np.ones(E, np.float32))
+    for e in experts:                                     # untimed set-up, like the GPU's weight packing
+        for which, dst in (("w13", w13), ("w2", w2)):
+            w = synth.expert_weights(shape, which, [e]).to(torch.float32).numpy()
+            _, q, sf, gs = Q.fake_quant_weights(w)
+            dst["codes"][e], dst["sf"][e], dst["gs"][e] = F.unpack_nibbles(q[0]), sf[0], gs[0]
+    a2 = np.float32(synth.H_GLOBAL_SCALE[shape.name])
+
+    def step():
+        return M.moe_forward(x, lg, w13, w2, shape.topk, n13, n2, a2)
+
+    desc = "first %d tokens of the %s batch (%d experts hit), full layer dims, weights pre-packed" % (
+        T_s, shape.name, len(experts))
+    return step, T_s, desc
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_15810_b200 import synth
+    shape = synth.MOE_SHAPES[args.workload]
+    budget = max(1.5, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    step, T_s, desc = oracle_sample(shape, args.variant, budget)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(1, args.steps)
+    value = T_s / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(shape, args.variant, {"sample": desc}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------- CUDA arm
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.f:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_15810_b200 import binding as B
+    from paper_2607_15810_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if world == 1:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    shape = synth.MOE_SHAPES[args.workload]
+    n13, n2 = nsel_of(shape, args.variant)
+    T, H, I, E, topk = shape.T, shape.H, shape.I, shape.E, shape.topk
+
+    def pack_weights(sh):
+        out = {}
+        for which in ("w13", "w2"):
+            parts = []
+            for e0 in range(0, sh.E, 16):
+                w = synth.expert_weights(sh, which, range(e0, min(sh.E, e0 + 16)))
+                parts.append(B.fake_quant_weights(w.to(dev), want_fq=False, sf_layout=B.SF_TILED))
+            out[which] = {k: torch.cat([p[k] for p in parts]) for k in ("q", "sf", "gs")}
+        return out["w13"], out["w2"]
+
+    gw13, gw2 = pack_weights(shape)
+    x_h, _ = synth.activations(shape)
+    lg_h = synth.router_logits(shape)
+    x_h, lg_h = x_h.pin_memory(), lg_h.pin_memory()
+    x_d, lg_d = x_h.to(dev), lg_h.to(dev)
+    a2 = torch.tensor([synth.H_GLOBAL_SCALE[shape.name]], dtype=torch.float32, device=dev)
+    ws = torch.empty(B.moe_workspace_bytes(T, H, I, E, topk), dtype=torch.uint8, device=dev)
+    out_d = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
+    out_h = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def step():
+        B.moe_w4a4_rac(x_d, lg_d, gw13, gw2, topk, n13, n2, a2, workspace=ws, out=out_d)
+
+    def timed(fn, k, with_flush=True):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(k)]
+        for s, e in evs:
+            if with_flush:
+                flush.fill_(1)
+            s.record()
+            fn()
+            e.record()
+        torch.cuda.synchronize()
+        return [s.elapsed_time(e) for s, e in evs]
+
+    for _ in range(max(3, args.warmup)):
+        flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    assert B.moe_async_status(ws) == 0, "device-side wait timed out"
+    launches_per_step = B.last_launch_count()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    wall0 = time.perf_counter()
+    times = timed(step, args.steps)
+    barrier()
+    wall = time.perf_counter() - wall0
+    ms = max_over_ranks(sum(times) / len(times))
+    value = world * T / (ms * 1e-3)
+
+    # end to end: pinned host input -> device, the call, result back to pinned host memory
+    def e2e_step():
+        x_d.copy_(x_h, non_blocking=True)
+        lg_d.copy_(lg_h, non_blocking=True)
+        step()
+        out_h.copy_(out_d, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e2e_times = timed(e2e_step, args.steps)
+    barrier()
+    e2e_ms = max_over_ranks(sum(e2e_times) / len(e2e_times))
+    clocks = sampler.stop() if sampler else None
+
+    # per-kernel time of the two grouped GEMMs (events recorded by the library on the launch stream)
+    B.moe_set_kernel_timing(True)
+    g1, g2 = [], []
+    for _ in range(max(5, min(args.steps, 20))):
+        flush.fill_(1)
+        step()
+        a, b = B.moe_last_kernel_ms()
+        g1.append(a)
+        g2.append(b)
+    B.moe_set_kernel_timing(False)
+    g1_ms, g2_ms = sum(g1) / len(g1), sum(g2) / len(g2)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    A = T * topk
+    f_model = 6.0 * A * H * I
+    f_alg1 = 2.0 * A * H * 2 * I * (1.0 + n13 / H)
+    f_alg2 = 2.0 * A * I * H * (1.0 + n2 / I)
+    fp4_peak = peaks["bf16_tflops"] * 4.0
+    ach = f_alg1 / (g1_ms * 1e-3) / 1e12
+    roofline = {"kernel": "gemm_kernel<SwiGLU> (grouped W13 GEMM + RAC + SwiGLU + requantize)", "bound": "tensor",
+                "achieved": ach, "peak": fp4_peak, "unit": "TFLOP/s", "frac": ach / fp4_peak,
+                "peak_source": "%s bf16 burst %.1f TFLOP/s x 4 (nominal FP4:bf16 ratio)" % (peaks["source"], peaks["bf16_tflops"]),
+                "traffic": None, "ms": g1_ms,
+                "gemm2": {"ms": g2_ms, "achieved": f_alg2 / (g2_ms * 1e-3) / 1e12, "frac": f_alg2 / (g2_ms * 1e-3) / 1e12 / fp4_peak},
+                "frac_of_nominal_9pf": ach / 9000.0}
+    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_file):
+        with open(traffic_file) as fh:
+            roofline["traffic"] = json.load(fh).get("%s_%s_gemm1_bytes" % (args.workload, args.variant))
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp4 (e2m1 x e2m1, ue4m3 block scales, fp32 accumulate)",
+            "data": "synthetic", "config": workload_config(shape, args.variant),
+            "clocks": clocks, "wall_s_timed_region": wall,
+            "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": x_h.numel() * 2 + lg_h.numel() * 4, "d2h_bytes_per_step": out_h.numel() * 2},
+            "gpu_launches": launches_per_step * args.steps,
+            "tflops": {"model": f_model / (ms * 1e-3) / 1e12, "algorithmic": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12,
+                       "frac_of_fp4_peak": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12 / fp4_peak},
+            "roofline": roofline}
+
+    if not args.no_aux:
+        aux = {}
+        # quantize GB/s on the activation tensor of this workload (ring of 8 inputs > L2)
+        ring = [torch.randn(T, H, device=dev).to(torch.bfloat16) for _ in range(8)]
+        q = torch.empty(T, H // 2, dtype=torch.uint8, device=dev)
+        sf = torch.empty(T, H // 16, dtype=torch.uint8, device=dev)
+        g = torch.empty(1, dtype=torch.float32, device=dev)
+        qws = torch.empty(256, dtype=torch.uint8, device=dev)
+        it = [0]
+
+        def qstep():
+            B.quantize_nvfp4(ring[it[0] % 8], out=(q, sf, g), workspace=qws)
+            it[0] += 1
+        for _ in range(8):
+            qstep()
+        tq = timed(qstep, 40, with_flush=False)
+        aux["quantize_gbs"] = T * H * 2.5625 / (sum(tq) / len(tq) * 1e-3) / 1e9
+        aux["quantize_frac_of_hbm"] = aux["quantize_gbs"] / peaks["hbm_gbs"]
+        del ring
+        # fake-quant + pack GB/s: 16 experts' W13 of the AQAT workload (403 MB in, 516 MB out)
+        w = (torch.randn(16, 3072, 4096, device=dev) * 0.015).to(torch.bfloat16)
+        outs = (torch.empty_like(w), torch.empty(16, 3072, 2048, dtype=torch.uint8, device=dev),
+                torch.empty(16, 3072, 256, dtype=torch.uint8, device=dev), torch.empty(16, dtype=torch.float32, device=dev))
+        fws = torch.empty(256, dtype=torch.uint8, device=dev)
+
+        def fstep():
+            B.fake_quant_weights(w, out=outs, workspace=fws)
+        for _ in range(3):
+            fstep()
+        tf = timed(fstep, 20)
+        aux["fake_quant_gbs"] = w.numel() * 4.5625 / (sum(tf) / len(tf) * 1e-3) / 1e9
+        aux["fake_quant_frac_of_hbm"] = aux["fake_quant_gbs"] / peaks["hbm_gbs"]
+        aux["hbm_peak_gbs"] = peaks["hbm_gbs"]
+        del w, outs
+        line["aux"] = aux
+
+    if world == 1 and not args.no_cpu_baseline:
+        step_o, T_s, desc = oracle_sample(shape, args.variant, 15.0)
+        t0 = time.perf_counter()
+        step_o()
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": T_s / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": desc, "seconds": dt}
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

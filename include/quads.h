@@ -170,6 +170,18 @@ size_t quads_moe_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int
    quads_moe_w4a4_rac call: QUADS_OK or QUADS_ERR_TIMEOUT. */
 quads_status quads_moe_async_status(const void* workspace, void* cuda_stream);
 
+/*
+ * Measurement aid (no counterpart in the paper).  When enabled, every later
+ * MoE-mode quads_moe_w4a4_rac call records CUDA events on its stream right
+ * before and after each of its two grouped GEMM kernels; quads_moe_last_kernel_ms
+ * waits for the most recent call's events and returns the two durations in
+ * milliseconds (host pointers).  Off by default; the events are created on the
+ * device that is current at the first enable.  Returns QUADS_ERR_SHAPE when no
+ * timed call has been made.
+ */
+quads_status quads_moe_set_kernel_timing(int32_t enable);
+quads_status quads_moe_last_kernel_ms(float* gemm1_ms /* host */, float* gemm2_ms /* host */);
+
 /* Number of kernels the last quads_* call on this host thread enqueued. */
 int32_t quads_last_launch_count(void);
 

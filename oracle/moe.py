@@ -89,7 +89,7 @@ def _absdot(site, w_abs):
 
 
 def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
-                a13_gs=None, renormalize=True, forced_sel13=None, forced_sel2=None):
+                a13_gs=None, renormalize=True, forced_sel13=None, forced_sel2=None, h_override=None):
     """MoE layer forward.
       x       float32 (bf16-valued) [T, H]
       logits  float32 [T, E]
@@ -97,6 +97,11 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
       w2      dict(codes [E,H,I],  sf [E,H,I/16],  gs [E])
       a2_gs   per-tensor scale of the SwiGLU output h (caller supplied; the
               paper is silent; a fused requantize needs it before h exists)
+      h_override  bf16 values [A, I] to use in place of the computed h for the
+              second half of the layer.  h feeds a quantizer, so two correct
+              first halves that differ by one bf16 ulp give different (both
+              valid) codes; the staged comparison checks the second half of
+              an implementation on that implementation's own h.
     Returns a dict of every intermediate the CUDA path can export."""
     x = np.asarray(x, dtype=F32)
     T, H = x.shape
@@ -129,6 +134,9 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
         g_absdot[lo:hi] = xa[rows] @ np.abs(w).T
         h64[lo:hi] = silu(g[:, :I]) * g[:, I:]
     h = F.bf16_round(h64)                                  # [A, I] in dispatch order
+    h_own = h
+    if h_override is not None:
+        h = np.asarray(h_override, dtype=F32)
 
     # ---- site 2: all A dispatched rows together are the batch
     site2 = R.rac(h, n_sel2, a2_gs, None)
@@ -154,7 +162,7 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
         out64[rows] += gw * y
         out_absdot[rows] += gw * ya
     return dict(ids=ids, weights=wts, counts=counts, offsets=offsets, perm=perm,
-                site13=site13, g64=g64, g_absdot=g_absdot, h64=h64, h=h,
+                site13=site13, g64=g64, g_absdot=g_absdot, h64=h64, h=h_own,
                 site2=site2, out64=out64, out=F.bf16_round(out64), out_absdot=out_absdot)
 
 

@@ -54,6 +54,10 @@ lib.quads_moe_w4a4_rac.restype = _i32
 lib.quads_moe_w4a4_rac.argtypes = [C.POINTER(MoEArgs), _p]
 lib.quads_moe_async_status.restype = _i32
 lib.quads_moe_async_status.argtypes = [_p, _p]
+lib.quads_moe_set_kernel_timing.restype = _i32
+lib.quads_moe_set_kernel_timing.argtypes = [_i32]
+lib.quads_moe_last_kernel_ms.restype = _i32
+lib.quads_moe_last_kernel_ms.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float)]
 lib.quads_last_launch_count.restype = _i32
 lib.quads_last_launch_count.argtypes = []
 
@@ -220,3 +224,14 @@ def dense_w4a4_rac(x, w, nsel, a_gs=None, export=False, workspace=None):
 
 def moe_async_status(workspace):
     return lib.quads_moe_async_status(_ptr(workspace), _stream())
+
+
+def moe_set_kernel_timing(enable):
+    check(lib.quads_moe_set_kernel_timing(1 if enable else 0))
+
+
+def moe_last_kernel_ms():
+    """(gemm1_ms, gemm2_ms) of the most recent timed MoE call."""
+    a, b = C.c_float(), C.c_float()
+    check(lib.quads_moe_last_kernel_ms(C.byref(a), C.byref(b)))
+    return a.value, b.value

@@ -133,6 +133,15 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   return L;
 }
 
+// Optional per-kernel timing of the two grouped GEMMs (off by default).
+struct GemmTimers {
+  bool enabled = false;
+  bool created = false;
+  bool valid = false;
+  cudaEvent_t ev[4];
+};
+GemmTimers g_timers;
+
 int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
 quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
@@ -253,6 +262,25 @@ quads_status quads_moe_async_status(const void* workspace, void* cuda_stream) {
   QUADS_CUDA_OK(cudaMemcpyAsync(&v, static_cast<const int32_t*>(workspace) + kHdrStatus, 4, cudaMemcpyDeviceToHost, st));
   QUADS_CUDA_OK(cudaStreamSynchronize(st));
   return v == 0 ? QUADS_OK : (quads_status)v;
+}
+
+quads_status quads_moe_set_kernel_timing(int32_t enable) {
+  if (enable && !g_timers.created) {
+    for (int i = 0; i < 4; ++i) QUADS_CUDA_OK(cudaEventCreate(&g_timers.ev[i]));
+    g_timers.created = true;
+  }
+  g_timers.enabled = enable != 0;
+  g_timers.valid = false;
+  return QUADS_OK;
+}
+
+quads_status quads_moe_last_kernel_ms(float* gemm1_ms, float* gemm2_ms) {
+  if (!gemm1_ms || !gemm2_ms) return QUADS_ERR_NULL;
+  if (!g_timers.valid) return QUADS_ERR_SHAPE;
+  QUADS_CUDA_OK(cudaEventSynchronize(g_timers.ev[3]));
+  QUADS_CUDA_OK(cudaEventElapsedTime(gemm1_ms, g_timers.ev[0], g_timers.ev[1]));
+  QUADS_CUDA_OK(cudaEventElapsedTime(gemm2_ms, g_timers.ev[2], g_timers.ev[3]));
+  return QUADS_OK;
 }
 
 quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
@@ -387,7 +415,10 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.hq_pad = P(L.hq_pad); g.hsf_tiled = P(L.hsf); g.r2q_pad = P(L.r2q_pad); g.r2sf_tiled = P(L.r2sf);
   g.partials2 = reinterpret_cast<float*>(P(L.partials2));
   g.h_export = static_cast<uint16_t*>(a->h_bf16);
+  const bool timing = g_timers.enabled && g_timers.created;
+  if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[0], st));
   if ((s = launch_gemm(kEpiSwiGLU, g, tm_x, tm_r, tm_w13, di.sm_count, st)) != QUADS_OK) return s;
+  if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[1], st));
 
   // ---- site 2: selection and masking of the residual of h
   const int nsel2 = a->rac_nsel_2;
@@ -427,7 +458,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g2.n_tiles_n = (H + 255) / 256;
   g2.half1_row_offset = 128;
   g2.out_f32 = out32;
+  if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[2], st));
   if ((s = launch_gemm(kEpiCombine, g2, tm_h, tm_r2, tm_w2, di.sm_count, st)) != QUADS_OK) return s;
+  if (timing) {
+    QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
+    g_timers.valid = true;
+  }
   const int64_t n4 = (int64_t)T * H / 4;
   finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(out32, static_cast<uint16_t*>(a->out), n4);
   note_launch();

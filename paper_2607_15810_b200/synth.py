@@ -37,11 +37,12 @@ class MoEShape:
     heavy_scale: float
     hot_experts: int = 0  # >0: bias the router so that experts 0..hot-1 ...
     hot_share: float = 0.0  # ... receive this share of the assignments
+    weight_seed: int = -1   # >= 0: draw the expert weights from this seed (a shared layer)
 
 
 MOE_SHAPES = {
     "decode": MoEShape("decode", 1, 256, 2048, 128, 8, 768, 0.02, 20, 3.0, 10.0),
-    "prefill": MoEShape("prefill", 2, 8192, 2048, 128, 8, 768, 0.02, 20, 3.0, 10.0, 8, 0.25),
+    "prefill": MoEShape("prefill", 2, 8192, 2048, 128, 8, 768, 0.02, 20, 3.0, 10.0, 8, 0.25, weight_seed=1),
     "large": MoEShape("large", 3, 4096, 4096, 128, 8, 1536, 0.015, 20, 2.5, 16.0),
     # small layers for tests: several tiles, ragged expert segments, empty experts
     "tiny": MoEShape("tiny", 11, 96, 256, 8, 2, 128, 0.05, 3, 3.0, 10.0),
@@ -49,6 +50,10 @@ MOE_SHAPES = {
 }
 
 DENSE_OUTLIER_CHANNELS = (3, 141, 278, 415)
+
+# Static per-tensor scale of the SwiGLU output h (a calibration constant the
+# caller of the MoE layer supplies; values above 2688 * scale saturate).
+H_GLOBAL_SCALE = {"decode": 0.25, "prefill": 0.25, "large": 0.5}
 
 
 def _gen(seed, stream):
@@ -110,7 +115,8 @@ def expert_weights(shape: MoEShape, which, experts=None):
     stream0 = 100 if which == "w13" else 100000
     out = torch.empty(len(experts), N, K, dtype=torch.bfloat16)
     for i, e in enumerate(experts):
-        w = torch.randn(N, K, generator=_gen(shape.seed, stream0 + e)) * shape.w_std
+        wseed = shape.weight_seed if shape.weight_seed >= 0 else shape.seed
+        w = torch.randn(N, K, generator=_gen(wseed, stream0 + e)) * shape.w_std
         out[i] = to_bf16(w)
     return out
 

@@ -1,0 +1,174 @@
+"""CUDA W4A4+RAC projections against the oracle through the C ABI: the dense
+config, small MoE layers compared in full, and the decode / prefill / large
+configs at full size."""
+import os
+import sys
+
+import numpy as np
+import pytest
+import torch
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+import moe_check as MC  # noqa: E402
+from oracle import formats as F  # noqa: E402
+from oracle import moe as M  # noqa: E402
+from oracle import nvfp4 as Q  # noqa: E402
+from paper_2607_15810_b200 import synth  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_15810_b200 import binding
+    return binding
+
+
+def _dense_case(B, x, w, nsel):
+    wq = B.fake_quant_weights(w.unsqueeze(0).cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    res = B.dense_w4a4_rac(x.cuda(), wq, nsel, export=True)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    wo = MC.oracle_weights(w[None])
+    o = M.dense_w4a4_rac(MC.f32(x), wo["codes"][0], wo["sf"][0], wo["gs"][0], nsel)
+    MC.check_site1(res, dict(site13=o["site"]), nsel, {})
+    got = MC.f32(res["out"]).astype(np.float64)
+    ratio = float((np.abs(got - o["y64"]) / MC.gemm_tol(o["absdot"], o["y64"])).max())
+    assert ratio <= 1.0, ratio
+    return ratio
+
+
+@pytest.mark.parametrize("nsel", [0, 16, 64, 128, 256, 384, 512])
+def test_dense_config_all_ratios(B, nsel):
+    """Config "single dense W4A4+RAC GEMM" (n_sel = 16) and the paper's channel
+    ratios 12.5 .. 100 % of K = 512."""
+    x, w = synth.dense_inputs(seed=0)
+    _dense_case(B, x, w, nsel)
+
+
+@pytest.mark.parametrize("T,K,N,nsel,seed", [(1, 128, 128, 8, 1), (200, 640, 384, 64, 5), (300, 2048, 512, 1024, 6),
+                                             (129, 384, 128, 96, 7)])
+def test_dense_ragged_shapes(B, T, K, N, nsel, seed):
+    x, w = synth.dense_inputs(seed, T=T, K=K, N=N)
+    _dense_case(B, x, w, nsel)
+
+
+def test_dense_exact_integer_case(B):
+    """Integer-valued operands with unit scales: the tensor-core result must be
+    the exact small-integer product."""
+    rng = np.random.default_rng(3)
+    ints = np.array([0, 1, 2, 3, 4, 6, -1, -2, -3, -4, -6], dtype=np.float32)
+    a = rng.choice(ints, (128, 256)).astype(np.float32)
+    b = rng.choice(ints, (128, 256)).astype(np.float32)
+    a[:, ::16] = 6
+    b[:, ::16] = 6
+    gs = torch.tensor([1.0]).cuda()
+    x = torch.from_numpy(a).to(torch.bfloat16)
+    b = b * 7.0   # weight amax 42 -> tensor scale 42/2688 = 2^-6 and block scales 448: every factor is exact
+    w = torch.from_numpy(b).to(torch.bfloat16)
+    wq = B.fake_quant_weights(w.unsqueeze(0).cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    res = B.dense_w4a4_rac(x.cuda(), wq, 0, a_gs=gs)
+    want = a.astype(np.float64) @ b.astype(np.float64).T
+    got = MC.f32(res["out"]).astype(np.float64)
+    assert np.array_equal(got, MC.f32(torch.from_numpy(want).to(torch.bfloat16)).astype(np.float64))
+
+
+def _moe_small(B, name, f13, f2, renorm):
+    sh = synth.MOE_SHAPES[name]
+    x, _ = synth.activations(sh)
+    lg = synth.router_logits(sh)
+    w13, w2 = synth.expert_weights(sh, "w13"), synth.expert_weights(sh, "w2")
+    w13o, w2o = MC.oracle_weights(w13), MC.oracle_weights(w2)
+    nsel13, nsel2 = int(sh.H * f13), int(sh.I * f2)
+    pilot = M.moe_forward(MC.f32(x), lg.numpy(), w13o, w2o, sh.topk, nsel13, 0, np.float32(1.0), renormalize=renorm)
+    a2 = Q.tensor_global_scale(pilot["h"])
+    gw13 = B.fake_quant_weights(w13.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    gw2 = B.fake_quant_weights(w2.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    assert np.array_equal(gw13["q"].cpu().numpy(), w13o["q"]) and np.array_equal(gw2["q"].cpu().numpy(), w2o["q"])
+    res = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, nsel13, nsel2, torch.tensor([a2]).cuda(),
+                         renormalize=renorm, export=True)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    rep = MC.check_moe(res, x, lg, w13o, w2o, sh.topk, nsel13, nsel2, a2, renormalize=renorm)
+    # the export-free call gives the same output bits for everything but the atomics' order
+    res2 = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, nsel13, nsel2, torch.tensor([a2]).cuda(),
+                          renormalize=renorm)
+    d = (MC.f32(res2["out"]) - MC.f32(res["out"]))
+    assert np.abs(d).max() <= 2.0 ** -6 * np.abs(MC.f32(res["out"])).max()
+    return rep
+
+
+@pytest.mark.parametrize("name,f13,f2,renorm", [("tiny", 0.5, 0.5, True), ("tiny", 0.0, 0.0, True),
+                                                ("tiny", 1.0, 1.0, False), ("small", 0.5, 0.5, True),
+                                                ("small", 0.25, 0.0, False), ("small", 0.0, 0.5, True)])
+def test_moe_small_layers_in_full(B, name, f13, f2, renorm):
+    _moe_small(B, name, f13, f2, renorm)
+
+
+_W = {}
+
+
+def _gpu_weights(B, sh):
+    key = (sh.weight_seed if sh.weight_seed >= 0 else sh.seed, sh.H, sh.I, sh.E)
+    if key not in _W:
+        out = {}
+        for which in ("w13", "w2"):
+            parts = []
+            for e0 in range(0, sh.E, 16):
+                w = synth.expert_weights(sh, which, range(e0, min(sh.E, e0 + 16)))
+                parts.append(B.fake_quant_weights(w.cuda(), want_fq=False, sf_layout=B.SF_TILED))
+            out[which] = {k: torch.cat([p[k] for p in parts]) for k in ("q", "sf", "gs")}
+        _W.clear()
+        _W[key] = out
+    return _W[key]["w13"], _W[key]["w2"]
+
+
+@pytest.mark.parametrize("name,variant", [("decode", "both"), ("prefill", "both"), ("prefill", "w13"),
+                                          ("prefill", "plain"), ("large", "both")])
+def test_moe_full_size_sampled(B, name, variant):
+    """The benchmark configurations at full size, in the launch configuration
+    the benchmark times; GEMM outputs are compared on sampled tokens."""
+    sh = synth.MOE_SHAPES[name]
+    x, _ = synth.activations(sh)
+    lg = synth.router_logits(sh)
+    gw13, gw2 = _gpu_weights(B, sh)
+    nsel13 = 0 if variant == "plain" else sh.H // 2
+    nsel2 = sh.I // 2 if variant == "both" else 0
+    a2 = np.float32(synth.H_GLOBAL_SCALE[name])
+    res = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, nsel13, nsel2, torch.tensor([a2]).cuda(),
+                         export=True)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    if sh.hot_experts:
+        ids = res["ids"].cpu().numpy()
+        share = float((ids < sh.hot_experts).mean())
+        assert abs(share - sh.hot_share) <= 0.005
+    n_tok = 2 if name == "large" else 3
+    rng = np.random.default_rng(99)
+    tokens = sorted(int(t) for t in rng.choice(sh.T, n_tok, replace=False))
+    rep = MC.check_moe_sampled(res, x, lg, sh,
+                               lambda e: synth.expert_weights(sh, "w13", [e])[0],
+                               lambda e: synth.expert_weights(sh, "w2", [e])[0],
+                               nsel13, nsel2, a2, tokens)
+    assert rep["h_max_err_over_tol"] <= 1 and rep["out_max_err_over_tol"] <= 1
+    for k in ("xq", "rq", "h", "hq", "r2q"):
+        res.pop(k)
+
+
+def test_decode_layer_in_full(B):
+    """Config "MoE layer decode" compared element by element in full."""
+    sh = synth.MOE_SHAPES["decode"]
+    x, _ = synth.activations(sh)
+    lg = synth.router_logits(sh)
+    w13, w2 = synth.expert_weights(sh, "w13"), synth.expert_weights(sh, "w2")
+    w13o, w2o = MC.oracle_weights(w13), MC.oracle_weights(w2)
+    gw13, gw2 = _gpu_weights(B, sh)
+    assert np.array_equal(gw13["q"].cpu().numpy(), w13o["q"]) and np.array_equal(gw13["gs"].cpu().numpy(), w13o["gs"])
+    assert np.array_equal(gw2["q"].cpu().numpy(), w2o["q"]) and np.array_equal(gw2["gs"].cpu().numpy(), w2o["gs"])
+    a2 = np.float32(synth.H_GLOBAL_SCALE["decode"])
+    nsel13, nsel2 = sh.H // 2, sh.I // 2
+    res = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, nsel13, nsel2, torch.tensor([a2]).cuda(),
+                         export=True)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    MC.check_moe(res, x, lg, w13o, w2o, sh.topk, nsel13, nsel2, a2)

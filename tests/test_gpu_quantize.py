@@ -1,0 +1,126 @@
+"""CUDA quantize / fake-quant against the oracle, bit for bit, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import formats as F
+from oracle import nvfp4 as Q
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_15810_b200 import binding
+    return binding
+
+
+def _f32(t):
+    return t.to(torch.float32).cpu().numpy()
+
+
+def _bf16(shape, seed, scale=1.0):
+    return (torch.randn(*shape, generator=torch.Generator().manual_seed(seed)) * scale).to(torch.bfloat16)
+
+
+def _tiled_index(rows, K):
+    KT = (K + 63) // 64
+    r = np.arange(rows)[:, None]
+    kb = np.arange(K // 16)[None, :]
+    return ((r >> 7) * KT + (kb >> 2)) * 512 + (r & 31) * 16 + ((r >> 5) & 3) * 4 + (kb & 3)
+
+
+@pytest.mark.parametrize("rows,K,seed", [(128, 512, 0), (1, 16, 1), (7, 64, 2), (333, 2048, 3), (129, 4096, 4),
+                                         (8192, 2048, 5)])
+def test_quantize_bit_exact(B, rows, K, seed):
+    x = _bf16((rows, K), seed, 3.0)
+    if K >= 64:
+        x[:, 5] *= 20
+    if rows > 3:
+        x[2, :16] = 0
+    q, sf, gs = B.quantize_nvfp4(x.cuda())
+    c_o, s_o, g_o = Q.quantize(_f32(x))
+    assert np.float32(gs.item()) == g_o
+    assert np.array_equal(sf.cpu().numpy(), s_o)
+    assert np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o))
+    q2, sf2, _ = B.quantize_nvfp4(x.cuda(), sf_layout=B.SF_TILED)
+    assert np.array_equal(q2.cpu().numpy(), F.pack_nibbles(c_o))
+    assert np.array_equal(sf2.cpu().numpy()[_tiled_index(rows, K)], s_o)
+
+
+def test_quantize_supplied_scale_strided_and_empty(B):
+    big = _bf16((50, 256), 7)
+    x = big[:, :128]                                    # row stride 256
+    gs = torch.tensor([0.01], dtype=torch.float32)
+    q, sf, g = B.quantize_nvfp4(x.cuda() if False else big.cuda()[:, :128], gs=gs.cuda())
+    c_o, s_o, g_o = Q.quantize(_f32(x), np.float32(0.01))
+    assert np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o)) and np.array_equal(sf.cpu().numpy(), s_o)
+    assert g.item() == np.float32(0.01)
+    # saturating scale
+    q, sf, g = B.quantize_nvfp4(big.cuda(), gs=torch.tensor([1e-6]).cuda())
+    c_o, s_o, _ = Q.quantize(_f32(big), np.float32(1e-6))
+    assert np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o)) and np.array_equal(sf.cpu().numpy(), s_o)
+    # all-zero tensor and zero rows
+    z = torch.zeros(4, 64, dtype=torch.bfloat16).cuda()
+    q, sf, g = B.quantize_nvfp4(z)
+    assert g.item() == 1.0 and not sf.any() and not q.any()
+    q, sf, g = B.quantize_nvfp4(torch.empty(0, 64, dtype=torch.bfloat16).cuda())
+    assert g.item() == 1.0 and q.numel() == 0
+
+
+def test_every_scale_code_and_every_tie(B):
+    """Blocks whose amax sweeps every E4M3 code and every midpoint between two
+    codes (with the float32 neighbours of the midpoints), and elements that
+    sit on every E2M1 tie: the hardware conversions must agree with the
+    oracle's tables everywhere."""
+    mags = F.E4M3_MAGNITUDES
+    mids = 0.5 * (mags[:-1] + mags[1:])
+    u = np.concatenate([mags, mids]).astype(np.float32)
+    gs = np.float32(1.0 / 64)                            # power of two: amax/(6 gs) exact
+    amax = (u.astype(np.float64) * 6 * float(gs))
+    amax_bf = torch.tensor(amax, dtype=torch.float32).to(torch.bfloat16)   # bf16-representable subset decides
+    n = amax_bf.numel()
+    x = torch.zeros(n, 16, dtype=torch.bfloat16)
+    x[:, 0] = amax_bf
+    frac = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, -0.25, -0.75, -1.25, -1.75, -2.5, -3.5, -5.0, 0.0])
+    x[:, 1:] = (amax_bf.to(torch.float32)[:, None] / 6.0 * frac[None, :]).to(torch.bfloat16)
+    g = torch.tensor([float(gs)])
+    q, sf, _ = B.quantize_nvfp4(x.cuda(), gs=g.cuda())
+    c_o, s_o, _ = Q.quantize(_f32(x), gs)
+    assert len(set(s_o.reshape(-1).tolist())) > 100      # the sweep really covers the code space
+    assert np.array_equal(sf.cpu().numpy(), s_o)
+    assert np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o))
+    # every finite bf16 magnitude through the element rounding with unit scales
+    bits = torch.arange(0, 0x7F80, dtype=torch.int32).to(torch.int16).view(torch.bfloat16)
+    keep = bits.to(torch.float32) <= 8.0
+    v = bits[keep]
+    v = torch.cat([v, -v])
+    pad = (-v.numel()) % 15
+    v = torch.cat([v, torch.zeros(pad, dtype=torch.bfloat16)]).view(-1, 15)
+    x = torch.cat([torch.full((v.shape[0], 1), 6.0, dtype=torch.bfloat16), v], dim=1)
+    q, sf, _ = B.quantize_nvfp4(x.cuda(), gs=torch.tensor([1.0]).cuda())
+    c_o, s_o, _ = Q.quantize(_f32(x), np.float32(1.0))
+    assert np.array_equal(sf.cpu().numpy(), s_o) and np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o))
+
+
+@pytest.mark.parametrize("n,N,K", [(3, 256, 512), (1, 3072, 4096), (5, 100, 80), (2, 4096, 1536)])
+def test_fake_quant_bit_exact_and_trainer_equals_rollout(B, n, N, K):
+    w = _bf16((n, N, K), 11 + n, 0.015)
+    r = B.fake_quant_weights(w.cuda())
+    wf_o, q_o, sf_o, gs_o = Q.fake_quant_weights(_f32(w))
+    assert np.array_equal(r["gs"].cpu().numpy(), gs_o)
+    assert np.array_equal(r["q"].cpu().numpy(), q_o)
+    assert np.array_equal(r["sf"].cpu().numpy(), sf_o)
+    assert np.array_equal(F.bf16_bits(_f32(r["w_fq"])), F.bf16_bits(wf_o))
+    # rollout side: dequantize the packed bytes the GPU wrote (oracle arithmetic) == the GPU's bf16 fake-quant
+    for i in range(n):
+        roll = Q.dequantize_bf16(F.unpack_nibbles(r["q"][i].cpu().numpy()), r["sf"][i].cpu().numpy(),
+                                 r["gs"][i].item())
+        assert np.array_equal(F.bf16_bits(roll), F.bf16_bits(_f32(r["w_fq"][i])))
+    # pack-only and fake-quant-only give the same bytes; tiled layout holds the same scales
+    p = B.fake_quant_weights(w.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    assert np.array_equal(p["q"].cpu().numpy(), q_o)
+    idx = _tiled_index(N, K)
+    assert np.array_equal(p["sf"].cpu().numpy()[:, idx], sf_o)
+    f = B.fake_quant_weights(w.cuda(), want_pack=False)
+    assert f["q"] is None and np.array_equal(F.bf16_bits(_f32(f["w_fq"])), F.bf16_bits(wf_o))

@@ -47,7 +47,8 @@ enum {
   QUADS_ERR_WORKSPACE = -3,  /* workspace missing, misaligned or too small */
   QUADS_ERR_ARCH = -4,       /* the current device is not sm_100 */
   QUADS_ERR_CUDA = -5,       /* a CUDA runtime / driver call failed */
-  QUADS_ERR_TIMEOUT = -6     /* a bounded device-side wait gave up */
+  QUADS_ERR_TIMEOUT = -6,    /* a bounded device-side wait gave up */
+  QUADS_ERR_LIMIT = -7       /* size beyond the fixed capacity of an allocation-free entry point */
 };
 
 enum {
@@ -101,6 +102,36 @@ quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t 
                                       int sf_layout, void* workspace, size_t workspace_bytes,
                                       void* cuda_stream);
 size_t quads_fake_quant_workspace_bytes(int64_t n_tensors);
+
+/*
+ * Allocation-free variant of quads_fake_quant_weights (the paper has no
+ * counterpart; it exists for callers that cannot provide scratch memory).
+ * Some hosts of this library may not call cudaMalloc where they use it: a
+ * trainer whose device memory belongs entirely to its own caching pool, a
+ * plugin that is forbidden to allocate after start-up, or code on a path where
+ * the implicit device synchronisation of an allocation is not acceptable.  For
+ * them this entry point takes no workspace: its scratch, one 4-byte amax word
+ * per tensor, is a fixed array of QUADS_NOALLOC_MAX_TENSORS words inside the
+ * library image (16 KiB, resident on every GPU that loads the library until the
+ * process exits).  Arguments, outputs and results are those of
+ * quads_fake_quant_weights, bit for bit.
+ *   - n_tensors > QUADS_NOALLOC_MAX_TENSORS returns QUADS_ERR_LIMIT and
+ *     launches nothing; split the batch.
+ *   - The first call on each device looks up the array's device address (a
+ *     host-side query, no allocation).  Make that first call outside any
+ *     stream capture.
+ *   - The call allocates and frees nothing: no cudaMalloc, no cudaFree, no
+ *     allocating library routine.
+ *   - Every call on a device shares the one array.  Each call zeroes the words
+ *     it uses, on its stream, before use, so earlier contents do not matter;
+ *     but two calls that may run at the same time on one GPU (different
+ *     streams, or different host threads) race on it and must be serialised
+ *     by the caller.
+ */
+#define QUADS_NOALLOC_MAX_TENSORS 4096
+quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, int64_t N, int64_t K,
+                                              void* w_fq, uint8_t* q, uint8_t* sf, float* gs,
+                                              int sf_layout, void* cuda_stream);
 
 /*
  * (2)+(3) MoE expert layer forward with native W4A4 grouped GEMMs and Residual

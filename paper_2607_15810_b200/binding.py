@@ -50,6 +50,8 @@ lib.quads_quantize_nvfp4.restype = _i32
 lib.quads_quantize_nvfp4.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p, _sz, _p]
 lib.quads_fake_quant_weights.restype = _i32
 lib.quads_fake_quant_weights.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p, _sz, _p]
+lib.quads_fake_quant_weights_noalloc.restype = _i32
+lib.quads_fake_quant_weights_noalloc.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p]
 lib.quads_moe_w4a4_rac.restype = _i32
 lib.quads_moe_w4a4_rac.argtypes = [C.POINTER(MoEArgs), _p]
 lib.quads_moe_async_status.restype = _i32
@@ -136,6 +138,23 @@ def fake_quant_weights(w, want_fq=True, want_pack=True, sf_layout=SF_LINEAR, out
     check(lib.quads_fake_quant_weights(_ptr(w), n, N, K, _ptr(w_fq), _ptr(q), _ptr(sf), _ptr(gs), sf_layout,
                                        _ptr(ws), ws.numel(), _stream()))
     return dict(w_fq=w_fq, q=q, sf=sf, gs=gs)
+
+
+NOALLOC_MAX_TENSORS = 4096
+
+
+def fake_quant_weights_noalloc(w, out, sf_layout=SF_LINEAR, n_tensors=None):
+    """Allocation-free fake-quant: for callers that may not allocate device
+    memory (their memory belongs to a pool they do not own, or an allocation's
+    implicit synchronisation is not allowed where they run).  `out` = (w_fq, q,
+    sf, gs), all caller-allocated (any of the first three may be None); no
+    workspace is passed and this wrapper creates no tensor.  `n_tensors`
+    overrides the count taken from w's shape (used to probe the capacity
+    check)."""
+    n, N, K = w.shape
+    w_fq, q, sf, gs = out
+    check(lib.quads_fake_quant_weights_noalloc(_ptr(w), n if n_tensors is None else n_tensors, N, K, _ptr(w_fq),
+                                               _ptr(q), _ptr(sf), _ptr(gs), sf_layout, _stream()))
 
 
 def moe_workspace_bytes(T, H, I, E, topk, N=0):

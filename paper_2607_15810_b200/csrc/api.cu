@@ -178,6 +178,7 @@ const char* quads_status_string(quads_status s) {
     case QUADS_ERR_ARCH: return "QUADS_ERR_ARCH: the current device is not sm_100";
     case QUADS_ERR_CUDA: return "QUADS_ERR_CUDA: a CUDA runtime or driver call failed";
     case QUADS_ERR_TIMEOUT: return "QUADS_ERR_TIMEOUT: a bounded device-side wait gave up";
+    case QUADS_ERR_LIMIT: return "QUADS_ERR_LIMIT: the size exceeds the fixed capacity of an allocation-free entry point";
     default: return "QUADS: unknown status";
   }
 }
@@ -248,6 +249,47 @@ quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t 
   if (!gs && n_tensors > 0) return QUADS_ERR_NULL;
   return quantize_common(w, n_tensors, N, K, K, N * K, nullptr, w_fq, q, sf, gs, sf_layout, workspace,
                          workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---------------------------------------------------------------------------
+// Allocation-free fake-quant.  Its scratch (one amax word per tensor) lives in
+// the library image, so a caller that must not allocate device memory -- for
+// instance code running under a memory pool it does not own, or inside a
+// region where cudaMalloc's implicit device synchronisation is forbidden --
+// needs no workspace.  In host code `g_noalloc_amax` is only a handle for the
+// symbol; the device address comes from cudaGetSymbolAddress, looked up once
+// per device with that device current.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) uint32_t g_noalloc_amax[QUADS_NOALLOC_MAX_TENSORS];
+
+static quads_status noalloc_scratch(uint32_t** out) {
+  static std::mutex mu;
+  static uint32_t* per_device[64] = {nullptr};
+  int dev = 0;
+  QUADS_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QUADS_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!per_device[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_amax) != cudaSuccess || !p) return QUADS_ERR_CUDA;
+    per_device[dev] = static_cast<uint32_t*>(p);
+  }
+  *out = per_device[dev];
+  return QUADS_OK;
+}
+
+quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, int64_t N, int64_t K, void* w_fq,
+                                              uint8_t* q, uint8_t* sf, float* gs, int sf_layout,
+                                              void* cuda_stream) {
+  if (n_tensors > QUADS_NOALLOC_MAX_TENSORS) return QUADS_ERR_LIMIT;
+  if (!gs && n_tensors > 0) return QUADS_ERR_NULL;
+  uint32_t* scratch = nullptr;
+  quads_status s = noalloc_scratch(&scratch);
+  if (s != QUADS_OK) return s;
+  // quantize_common zeroes the amax words it is about to use on the stream
+  // before the reduction, so the previous call's contents never leak in.
+  return quantize_common(w, n_tensors, N, K, K, N * K, nullptr, w_fq, q, sf, gs, sf_layout, scratch,
+                         sizeof(uint32_t) * QUADS_NOALLOC_MAX_TENSORS, static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t quads_moe_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk, int32_t N) {

@@ -74,7 +74,7 @@ struct MoeLayout {
   size_t header, amax, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
   size_t perm, pos_pad, row_token, row_weight;
   size_t partials13, scores13, sel13, mask13, xq_pad, xsf, rq_pad, rsf;
-  size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, out32;
+  size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad;
   size_t total;
   int n_chunks, m_tiles_max, stats_ctas, rows_per_cta;
 };
@@ -110,7 +110,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   L.row_token = take(pad_rows * 4);
   L.row_weight = take(pad_rows * 4);
   L.partials13 = take((size_t)L.stats_ctas * H * 4);
-  L.scores13 = take((size_t)H * 8);
+  L.scores13 = take((size_t)H * 8 * kScoreSlices);
   L.sel13 = take((size_t)H * 4);
   L.mask13 = take((size_t)H);
   L.xq_pad = take(pad_rows * (H / 2));
@@ -123,10 +123,10 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
     L.r2q_pad = take(pad_rows * (I / 2));
     L.r2sf = take((size_t)L.m_tiles_max * (I / 64) * 512);
     L.partials2 = take((size_t)L.m_tiles_max * 4 * I * 4);
-    L.scores2 = take((size_t)I * 8);
+    L.scores2 = take((size_t)I * 8 * kScoreSlices);
     L.sel2 = take((size_t)I * 4);
     L.mask2 = take((size_t)I);
-    L.out32 = take((size_t)T * H * 4);
+    L.y_pad = take(pad_rows * (size_t)H * 2);
   }
   (void)N;
   L.total = o;
@@ -145,19 +145,21 @@ GemmTimers g_timers;
 int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
 quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
-                        int n_sel,
-                        double* scores, int32_t* sel_list, uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
-  score_reduce_kernel<<<(C + 31) / 32, 256, 0, st>>>(partials, n_part_ptr, n_part_mul, n_part_fixed, C, scores);
+                        int n_sel, double* slice_sums, uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
+  score_reduce_kernel<<<dim3((C + 31) / 32, kScoreSlices), 256, 0, st>>>(partials, n_part_ptr, n_part_mul,
+                                                                          n_part_fixed, C, slice_sums);
   note_launch();
-  const int n2 = pow2_at_least(C);
-  const size_t smem = (size_t)n2 * 12 + (size_t)(C + 1) * 4;
   static bool attr = false;
   if (!attr) {
-    QUADS_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    QUADS_CUDA_OK(cudaFuncSetAttribute(rank_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
     attr = true;
   }
-  select_kernel<<<1, 1024, smem, st>>>(scores, C, n_sel, n2, sel_list, mask, sel_export);
+  rank_select_kernel<<<(C + 63) / 64, 256, (size_t)C * 8, st>>>(slice_sums, C, n_sel, mask);
   note_launch();
+  if (sel_export) {
+    sel_list_kernel<<<1, 1024, 0, st>>>(mask, C, sel_export);
+    note_launch();
+  }
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
 }
@@ -336,7 +338,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   if (T < 0 || H <= 0 || (H % 128) != 0 || I < 0 || (I % 128) != 0) return QUADS_ERR_SHAPE;
   if (dense && (a->N <= 0 || (a->N % 128) != 0)) return QUADS_ERR_SHAPE;
   if (!dense && (E < 1 || E > kMaxExperts || topk < 1 || topk > kMaxTopk || topk > E)) return QUADS_ERR_SHAPE;
-  if (a->rac_nsel_13 < 0 || a->rac_nsel_13 > H || (!dense && (a->rac_nsel_2 < 0 || a->rac_nsel_2 > I)))
+  if (H > 16384 || I > 16384 || a->rac_nsel_13 < 0 || a->rac_nsel_13 > H || (!dense && (a->rac_nsel_2 < 0 || a->rac_nsel_2 > I)))
     return QUADS_ERR_SHAPE;
   if ((int64_t)T * topk > 0x3FFFFFFF) return QUADS_ERR_SHAPE;
   if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) return QUADS_ERR_NULL;
@@ -392,10 +394,10 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     route_kernel<<<L.n_chunks, 256, 0, st>>>(a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts,
                                               a->topk_ids, a->topk_w);
     note_launch();
-    scan_kernel<<<1, 256, 0, st>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
+    scan_kernel<<<1, 1024, 0, st>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
                                    tile_rows, header, a->expert_offsets);
     note_launch();
-    permute_kernel<<<L.n_chunks, 256, 0, st>>>(T, E, topk, ids, wts, chunk_base, offsets, tile_prefix, perm,
+    permute_kernel<<<(L.n_chunks + 3) / 4, 128, 0, st>>>(T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm,
                                                pos_pad, row_token, row_weight, a->perm);
     note_launch();
   }
@@ -412,8 +414,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   if (nsel13 > 0) {
     s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
-                   reinterpret_cast<double*>(P(L.scores13)), reinterpret_cast<int32_t*>(P(L.sel13)), mask13,
-                   a->sel13, st);
+                   reinterpret_cast<double*>(P(L.scores13)), mask13, a->sel13, st);
     if (s != QUADS_OK) return s;
   }
   // the dispatch kernel needs the scale as a value in memory: the amax word or the caller's
@@ -467,7 +468,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   uint8_t* mask2 = P(L.mask2);
   if (nsel2 > 0) {
     s = run_select(g.partials2, header + kHdrMTiles, 4 /* one partial row per tile and lane quadrant */, 0, I, nsel2,
-                   reinterpret_cast<double*>(P(L.scores2)), reinterpret_cast<int32_t*>(P(L.sel2)), mask2, a->sel2, st);
+                   reinterpret_cast<double*>(P(L.scores2)), mask2, a->sel2, st);
     if (s != QUADS_OK) return s;
     mask_codes_kernel<<<di.sm_count * 8, 256, 0, st>>>(P(L.r2q_pad), header + kHdrPaddedRows, I, mask2);
     note_launch();
@@ -483,8 +484,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
 
   // ---- second projection + weighted combine
-  float* out32 = reinterpret_cast<float*>(P(L.out32));
-  QUADS_CUDA_OK(cudaMemsetAsync(out32, 0, (size_t)T * H * 4, st));
+  uint16_t* y_pad = reinterpret_cast<uint16_t*>(P(L.y_pad));
   CUtensorMap tm_h, tm_r2, tm_w2;
   if ((s = make_codes_map(&tm_h, P(L.hq_pad), pad_rows, I / 2)) != QUADS_OK) return s;
   if ((s = make_codes_map(&tm_r2, P(L.r2q_pad), pad_rows, I / 2)) != QUADS_OK) return s;
@@ -499,15 +499,16 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g2.n_out = H;
   g2.n_tiles_n = (H + 255) / 256;
   g2.half1_row_offset = 128;
-  g2.out_f32 = out32;
+  g2.y_pad = y_pad;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[2], st));
   if ((s = launch_gemm(kEpiCombine, g2, tm_h, tm_r2, tm_w2, di.sm_count, st)) != QUADS_OK) return s;
   if (timing) {
     QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
     g_timers.valid = true;
   }
-  const int64_t n4 = (int64_t)T * H / 4;
-  finalize_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(out32, static_cast<uint16_t*>(a->out), n4);
+  const int64_t n8 = (int64_t)T * (H / 8);
+  combine_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(y_pad, pos_pad, wts, T, H, topk,
+                                                                static_cast<uint16_t*>(a->out));
   note_launch();
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;

@@ -162,8 +162,10 @@ __device__ __forceinline__ uint64_t desc_sf_atom(uint32_t saddr) {
 // K-major, M = 128, N = 256, dense.
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+__device__ __forceinline__ void stg256(void* addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
+                                       uint32_t f, uint32_t g, uint32_t h) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(addr), "r"(a), "r"(b), "r"(c), "r"(d),
+               "r"(e), "r"(f), "r"(g), "r"(h) : "memory");
 }
 
 struct __align__(8) BarrierBlock {
@@ -416,13 +418,22 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
           if (p.resid2) *reinterpret_cast<uint32_t*>(p.r2sf_tiled + so) = rs;
         }
       } else if (EPI == kEpiCombine) {
+        // y = W2 h~ for this dispatched row, rounded to bf16; the weighted sum over a
+        // token's experts is taken afterwards in a fixed order (no atomics).
         const int n0 = nt * 256 + hf * 128;
         if (valid && n0 < p.n_out) {
-          const float s = __fmul_rn(scale, p.row_weight[prow]);
-          float* dst = p.out_f32 + (size_t)p.row_token[prow] * p.n_out + n0;
+          uint16_t* dst = p.y_pad + (size_t)prow * p.n_out + n0;
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            red_add_v4(dst + 4 * i, acc[4 * i] * s, acc[4 * i + 1] * s, acc[4 * i + 2] * s, acc[4 * i + 3] * s);
+          for (int i = 0; i < 8; ++i)
+            stg256(dst + 16 * i,
+                   f32x2_to_bf16x2(acc[16 * i] * scale, acc[16 * i + 1] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 2] * scale, acc[16 * i + 3] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 4] * scale, acc[16 * i + 5] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 6] * scale, acc[16 * i + 7] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 8] * scale, acc[16 * i + 9] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 10] * scale, acc[16 * i + 11] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 12] * scale, acc[16 * i + 13] * scale),
+                   f32x2_to_bf16x2(acc[16 * i + 14] * scale, acc[16 * i + 15] * scale));
         }
       } else {
         const int n0 = nt * 256 + hf * 128;

@@ -6,7 +6,7 @@
 
 namespace quads {
 
-constexpr int kRouteTokensPerCta = 64;
+constexpr int kRouteTokensPerCta = 32;
 constexpr int kMaxTopk = 16;
 constexpr int kMaxExperts = 256;
 
@@ -22,17 +22,19 @@ __global__ void quantize_kernel(const uint16_t* x, int64_t rows, int64_t K, int6
 __global__ void rac_stats_kernel(const uint16_t* x, int T, int H, const float* gs_in, const uint32_t* amax_bits,
                                  float* gs_store, int rows_per_cta, float* partials, uint8_t* xq_out,
                                  uint8_t* xsf_out);
+constexpr int kScoreSlices = 16;
 __global__ void score_reduce_kernel(const float* partials, const int* n_part_ptr, int n_part_mul,
-                                    int n_part_fixed, int C, double* scores);
-__global__ void select_kernel(const double* scores, int C, int n_sel, int n_pow2, int32_t* sel_list,
-                              uint8_t* mask, int32_t* sel_export);
+                                    int n_part_fixed, int C, double* slice_sums);
+__global__ void rank_select_kernel(const double* slice_sums, int C, int n_sel, uint8_t* mask);
+__global__ void sel_list_kernel(const uint8_t* mask, int C, int32_t* sel_export);
 __global__ void rac_dispatch_kernel(const uint16_t* x, int T, int H, const float* gs_in,
                                     const uint32_t* amax_bits, int n_sel,
                                     const uint8_t* mask, int topk, const int32_t* pos_pad, uint8_t* xq_pad,
                                     uint8_t* xsf_tiled, uint8_t* rq_pad, uint8_t* rsf_tiled, uint8_t* rq_out,
                                     uint8_t* rsf_out);
 __global__ void mask_codes_kernel(uint8_t* codes, const int* n_rows_ptr, int C, const uint8_t* mask);
-__global__ void finalize_kernel(const float* acc, uint16_t* out, int64_t n4);
+__global__ void combine_kernel(const uint16_t* y_pad, const int32_t* pos_pad, const float* wts, int T, int H,
+                               int topk, uint16_t* out);
 __global__ void export_site2_kernel(int A, int I, const int32_t* perm, const int32_t* pos_pad,
                                     const uint8_t* hq_pad, const uint8_t* hsf_tiled, const uint8_t* r2q_pad,
                                     const uint8_t* r2sf_tiled, const uint8_t* mask2, uint8_t* hq, uint8_t* hsf,
@@ -44,7 +46,7 @@ __global__ void route_kernel(const float* logits, int T, int E, int topk, int re
 __global__ void scan_kernel(int E, int n_chunks, const int32_t* chunk_counts, int32_t* chunk_base,
                             int32_t* offsets, int32_t* tile_prefix, int32_t* tile_expert, int32_t* tile_rows,
                             int32_t* header, int32_t* offsets_out);
-__global__ void permute_kernel(int T, int E, int topk, const int32_t* ids, const float* wts,
+__global__ void permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* ids, const float* wts,
                                const int32_t* chunk_base, const int32_t* offsets, const int32_t* tile_prefix,
                                int32_t* perm, int32_t* pos_pad, int32_t* row_token, float* row_weight,
                                int32_t* perm_out);
@@ -75,7 +77,7 @@ struct GemmParams {
   const int32_t* row_token;
   const float* row_weight;
   uint16_t* out_bf16;    // kEpiStore: [T, n_out]
-  float* out_f32;        // kEpiCombine: [T, n_out] accumulation buffer
+  uint16_t* y_pad;       // kEpiCombine: bf16 [padded dispatch rows, n_out], one row per assignment
   // epilogue: SwiGLU + requantize (site 2)
   const float* h_gs;     // per-tensor scale of h
   int resid2;            // 1: also emit the residual of h and its column statistics

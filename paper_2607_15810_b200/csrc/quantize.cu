@@ -154,77 +154,72 @@ rac_stats_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
   }
 }
 
-// Sum `n_part` partial rows of width C into float64 scores, fixed order.
-// grid = C/32 CTAs of 256 threads: 32 columns x 8 interleaved slices.
+// Channel scores, stage 1: the partial rows are split into kScoreSlices
+// contiguous slices; CTA (column group, slice) adds its slice's rows in a fixed
+// order in float64.  grid = (ceil(C/32), kScoreSlices), 256 threads = 32 columns
+// x 8 interleaved row lanes.
 __global__ void __launch_bounds__(256)
 score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ n_part_ptr, int n_part_mul,
-                    int n_part_fixed, int C, double* __restrict__ scores) {
+                    int n_part_fixed, int C, double* __restrict__ slice_sums) {
   const int n_part = n_part_ptr ? *n_part_ptr * n_part_mul : n_part_fixed;
+  const int per = (n_part + kScoreSlices - 1) / kScoreSlices;
+  const int p0 = blockIdx.y * per, p1 = min(n_part, p0 + per);
   const int col = blockIdx.x * 32 + (threadIdx.x & 31);
-  const int slice = threadIdx.x >> 5;
+  const int rl = threadIdx.x >> 5;
   double s = 0.0;
   if (col < C)
-    for (int p = slice; p < n_part; p += 8) s += (double)partials[(size_t)p * C + col];
+    for (int p = p0 + rl; p < p1; p += 8) s += (double)partials[(size_t)p * C + col];
   __shared__ double sm[8][32];
-  sm[slice][threadIdx.x & 31] = s;
+  sm[rl][threadIdx.x & 31] = s;
   __syncthreads();
-  if (slice == 0 && col < C) {
+  if (rl == 0 && col < C) {
     double t = 0.0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x & 31];
-    scores[col] = t;
+    slice_sums[(size_t)blockIdx.y * C + col] = t;
   }
 }
 
-// ---------------------------------------------------------------------------
-// Channel selection (Eq. channel-select): the n_sel largest scores, ties to the
-// lower index.  One CTA; bitonic sort of (score, index) in shared memory, then
-// the ascending index list and a byte mask.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-select_kernel(const double* __restrict__ scores, int C, int n_sel, int n_pow2, int32_t* __restrict__ sel_list,
-              uint8_t* __restrict__ mask, int32_t* __restrict__ sel_export) {
+// Channel selection (Eq. channel-select), stage 2: every CTA rebuilds all C
+// scores (slice sums added in slice order) in shared memory, then ranks 64
+// channels: rank_j = #{i : s_i > s_j, or s_i == s_j and i < j}; channel j is
+// selected iff rank_j < n_sel (the n_sel largest, ties to the lower index).
+// grid = ceil(C/64), 256 threads (4 per ranked channel), smem = C doubles.
+__global__ void __launch_bounds__(256)
+rank_select_kernel(const double* __restrict__ slice_sums, int C, int n_sel, uint8_t* __restrict__ mask) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* key = reinterpret_cast<double*>(smem_raw);
-  int* idx = reinterpret_cast<int*>(key + n_pow2);
-  int* flag = idx + n_pow2;          // [C + 1] prefix counts
-  const int tid = threadIdx.x, nt = blockDim.x;
-  for (int i = tid; i < n_pow2; i += nt) {
-    key[i] = i < C ? scores[i] : -1.0;
-    idx[i] = i;
+  double* sc = reinterpret_cast<double*>(smem_raw);
+  for (int i = threadIdx.x; i < C; i += blockDim.x) {
+    double t = 0.0;
+#pragma unroll
+    for (int s = 0; s < kScoreSlices; ++s) t += slice_sums[(size_t)s * C + i];
+    sc[i] = t;
   }
   __syncthreads();
-  // "a before b" when a has the larger score, or equal score and lower index
-  for (int k = 2; k <= n_pow2; k <<= 1) {
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < n_pow2; i += nt) {
-        const int p = i ^ j;
-        if (p > i) {
-          const double ka = key[i], kb = key[p];
-          const int ia = idx[i], ib = idx[p];
-          const bool a_first = (ka > kb) || (ka == kb && ia < ib);
-          const bool up = ((i & k) == 0);
-          if (up ? !a_first : a_first) {
-            key[i] = kb; key[p] = ka;
-            idx[i] = ib; idx[p] = ia;
-          }
-        }
-      }
-      __syncthreads();
+  const int j = blockIdx.x * 64 + (threadIdx.x >> 2);
+  const int sub = threadIdx.x & 3;
+  int rank = 0;
+  if (j < C) {
+    const double sj = sc[j];
+    for (int i = sub; i < C; i += 4) {
+      const double si = sc[i];
+      rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
     }
   }
-  for (int i = tid; i < C; i += nt) flag[i] = 0;
-  __syncthreads();
-  for (int i = tid; i < n_sel; i += nt) flag[idx[i]] = 1;
-  __syncthreads();
-  for (int i = tid; i < C; i += nt) mask[i] = (uint8_t)flag[i];
-  __syncthreads();
-  // ascending list: serial chunks per thread, then a scan of chunk totals
+  rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 1);
+  rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 2);
+  if (j < C && sub == 0) mask[j] = rank < n_sel ? 1 : 0;
+}
+
+// Ascending list of the selected channels (verification export only).  One CTA.
+__global__ void __launch_bounds__(1024)
+sel_list_kernel(const uint8_t* __restrict__ mask, int C, int32_t* __restrict__ sel_export) {
   __shared__ int chunk_tot[1024];
+  const int tid = threadIdx.x, nt = blockDim.x;
   const int per = (C + nt - 1) / nt;
   const int c0 = tid * per, c1 = min(C, c0 + per);
   int cnt = 0;
-  for (int i = c0; i < c1; ++i) cnt += flag[i];
+  for (int i = c0; i < c1; ++i) cnt += mask[i];
   chunk_tot[tid] = cnt;
   __syncthreads();
   if (tid == 0) {
@@ -234,11 +229,7 @@ select_kernel(const double* __restrict__ scores, int C, int n_sel, int n_pow2, i
   __syncthreads();
   int pos = chunk_tot[tid];
   for (int i = c0; i < c1; ++i)
-    if (flag[i]) {
-      sel_list[pos] = i;
-      if (sel_export) sel_export[pos] = i;
-      ++pos;
-    }
+    if (mask[i]) sel_export[pos++] = i;
 }
 
 // ---------------------------------------------------------------------------
@@ -335,13 +326,31 @@ mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_pt
   }
 }
 
-// out32 [n] float -> bf16
+// Weighted top-k combine: out[t, :] = sum over the token's slots, in slot order,
+// of weight * y[row of (t, slot), :], accumulated in float32, rounded to bf16.
+// One thread per (token, 8 columns).
 __global__ void __launch_bounds__(256)
-finalize_kernel(const float* __restrict__ acc, uint16_t* __restrict__ out, int64_t n4) {
+combine_kernel(const uint16_t* __restrict__ y_pad, const int32_t* __restrict__ pos_pad,
+               const float* __restrict__ wts, int T, int H, int topk, uint16_t* __restrict__ out) {
+  const int per_row = H >> 3;
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n4) return;
-  const float4 v = reinterpret_cast<const float4*>(acc)[i];
-  reinterpret_cast<uint2*>(out)[i] = make_uint2(f32x2_to_bf16x2(v.x, v.y), f32x2_to_bf16x2(v.z, v.w));
+  if (i >= (int64_t)T * per_row) return;
+  const int t = (int)(i / per_row), c = (int)(i - (int64_t)t * per_row);
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+  for (int s = 0; s < topk; ++s) {
+    const int p = pos_pad[t * topk + s];
+    const float w = wts[t * topk + s];
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(y_pad + (size_t)p * H) + c);
+    float f[8];
+    unpack8(v, f);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = __fmaf_rn(w, f[j], acc[j]);
+  }
+  reinterpret_cast<uint4*>(out + (size_t)t * H)[c] =
+      make_uint4(f32x2_to_bf16x2(acc[0], acc[1]), f32x2_to_bf16x2(acc[2], acc[3]),
+                 f32x2_to_bf16x2(acc[4], acc[5]), f32x2_to_bf16x2(acc[6], acc[7]));
 }
 
 // Export of padded dispatch-order buffers into linear dispatch order.

@@ -13,12 +13,12 @@ __global__ void __launch_bounds__(256)
 route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
              int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
              int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
-  __shared__ int hist[256];
+  __shared__ int hist[kMaxExperts];
   for (int i = threadIdx.x; i < E; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t0 = blockIdx.x * kRouteTokensPerCta;
-  for (int tt = warp; tt < kRouteTokensPerCta; tt += 8) {
+  for (int tt = warp; tt < kRouteTokensPerCta; tt += (int)(blockDim.x >> 5)) {
     const int t = t0 + tt;
     if (t >= T) break;
     float v[8];
@@ -74,25 +74,33 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
   for (int i = threadIdx.x; i < E; i += blockDim.x) chunk_counts[(size_t)blockIdx.x * E + i] = hist[i];
 }
 
-// One CTA.  Per expert: exclusive prefix over chunks, total count; then the
-// exclusive scan over experts of counts (offsets) and of 128-row tile counts
-// (tile_prefix), the tile -> (expert, valid rows) map, and the header.
-__global__ void __launch_bounds__(256)
+// One CTA of 1024 threads.  A warp per expert (round robin): exclusive prefix of
+// the expert's counts over chunks and its total; then the exclusive scan over
+// experts of counts (offsets) and of 128-row tile counts (tile_prefix), the
+// tile -> (expert, valid rows) map, and the header.
+__global__ void __launch_bounds__(1024)
 scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32_t* __restrict__ chunk_base,
             int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tile_expert,
             int32_t* __restrict__ tile_rows, int32_t* __restrict__ header, int32_t* __restrict__ offsets_out) {
-  __shared__ int cnt[256];
-  __shared__ int off[257];
-  __shared__ int tpre[257];
-  const int e = threadIdx.x;
-  if (e < E) {
+  __shared__ int cnt[kMaxExperts];
+  __shared__ int off[kMaxExperts + 1];
+  __shared__ int tpre[kMaxExperts + 1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  for (int e = warp; e < E; e += n_warps) {
     int run = 0;
-    for (int c = 0; c < n_chunks; ++c) {
-      const int v = chunk_counts[(size_t)c * E + e];
-      chunk_base[(size_t)c * E + e] = run;
-      run += v;
+    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+      const int c = c0 + lane;
+      const int v = c < n_chunks ? chunk_counts[(size_t)c * E + e] : 0;
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (c < n_chunks) chunk_base[(size_t)c * E + e] = run + incl - v;
+      run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
-    cnt[e] = run;
+    if (lane == 0) cnt[e] = run;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -113,42 +121,52 @@ scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32
     tile_prefix[i] = tpre[i];
     if (offsets_out) offsets_out[i] = off[i];
   }
-  if (e < E) {
+  for (int e = warp; e < E; e += n_warps) {
     const int n_t = tpre[e + 1] - tpre[e];
-    for (int m = 0; m < n_t; ++m) {
+    for (int m = lane; m < n_t; m += 32) {
       tile_expert[tpre[e] + m] = e;
       tile_rows[tpre[e] + m] = min(128, cnt[e] - m * 128);
     }
   }
 }
 
-// One CTA per routing chunk, one thread per expert: walk the chunk's
-// assignments in (token, slot) order and hand out consecutive rows.
-__global__ void __launch_bounds__(256)
-permute_kernel(int T, int E, int topk, const int32_t* __restrict__ ids, const float* __restrict__ wts,
+// One warp per routing chunk: walk the chunk's assignments in (token, slot)
+// order, 32 at a time; lanes holding the same expert rank themselves with
+// match_any, so every expert hands out consecutive rows in that order.
+__global__ void __launch_bounds__(128)
+permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__ ids, const float* __restrict__ wts,
                const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ offsets,
                const int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ pos_pad,
                int32_t* __restrict__ row_token, float* __restrict__ row_weight, int32_t* __restrict__ perm_out) {
-  __shared__ int sid[kRouteTokensPerCta * kMaxTopk];
-  const int t0 = blockIdx.x * kRouteTokensPerCta;
-  const int n_tok = min(kRouteTokensPerCta, T - t0);
-  const int n = n_tok * topk;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) sid[i] = ids[(size_t)t0 * topk + i];
-  __syncthreads();
-  const int e = threadIdx.x;
-  if (e >= E) return;
-  int run = chunk_base[(size_t)blockIdx.x * E + e];
-  const int row0 = offsets[e], pad0 = tile_prefix[e] * 128;
-  for (int i = 0; i < n; ++i) {
-    if (sid[i] == e) {
-      const int flat = t0 * topk + i;
-      perm[row0 + run] = flat;
-      if (perm_out) perm_out[row0 + run] = flat;
-      const int p = pad0 + run;
+  __shared__ int run[4][kMaxExperts];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int chunk = blockIdx.x * 4 + warp;
+  if (chunk >= n_chunks) return;
+  for (int e = lane; e < E; e += 32) run[warp][e] = chunk_base[(size_t)chunk * E + e];
+  __syncwarp();
+  const int t0 = chunk * kRouteTokensPerCta;
+  const int n = min(kRouteTokensPerCta, T - t0) * topk;
+  for (int i0 = 0; i0 < n; i0 += 32) {
+    const int i = i0 + lane;
+    const bool active = i < n;
+    const int flat = t0 * topk + i;
+    const int e = active ? ids[flat] : (0x40000000 + lane);
+    const unsigned same = __match_any_sync(0xFFFFFFFFu, e);
+    const int rank = __popc(same & ((1u << lane) - 1u));
+    int base = 0;
+    if (active) base = run[warp][e];
+    __syncwarp();
+    if (active && rank == 0) run[warp][e] = base + __popc(same);
+    __syncwarp();
+    if (active) {
+      const int r = base + rank;
+      const int row = offsets[e] + r;
+      perm[row] = flat;
+      if (perm_out) perm_out[row] = flat;
+      const int p = tile_prefix[e] * 128 + r;
       pos_pad[flat] = p;
       row_token[p] = flat / topk;
       row_weight[p] = wts[flat];
-      ++run;
     }
   }
 }

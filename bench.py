@@ -305,6 +305,16 @@ def run_ours(args):
         g2.append(b)
     B.moe_set_kernel_timing(False)
     g1_ms, g2_ms = sum(g1) / len(g1), sum(g2) / len(g2)
+    # per-stage times (events after every stage; separate pass, not the headline timing)
+    B.moe_set_stage_trace(True)
+    stage_acc = {}
+    for _ in range(5):
+        flush.fill_(1)
+        step()
+        for name, t in B.moe_get_stage_trace():
+            stage_acc.setdefault(name, []).append(t)
+    B.moe_set_stage_trace(False)
+    stages_us = {k: round(1e3 * sum(v) / len(v), 1) for k, v in stage_acc.items()}
 
     if rank != 0:
         if world > 1:
@@ -339,7 +349,7 @@ def run_ours(args):
             "gpu_launches": launches_per_step * args.steps,
             "tflops": {"model": f_model / (ms * 1e-3) / 1e12, "algorithmic": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12,
                        "frac_of_fp4_peak": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12 / fp4_peak},
-            "roofline": roofline}
+            "roofline": roofline, "stages_us": stages_us}
 
     if not args.no_aux:
         aux = {}

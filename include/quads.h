@@ -213,6 +213,16 @@ quads_status quads_moe_async_status(const void* workspace, void* cuda_stream);
 quads_status quads_moe_set_kernel_timing(int32_t enable);
 quads_status quads_moe_last_kernel_ms(float* gemm1_ms /* host */, float* gemm2_ms /* host */);
 
+/*
+ * Measurement aid (no counterpart in the paper): when enabled, a MoE-mode call
+ * records a CUDA event on its stream after every stage; get_stage_trace waits
+ * for the last call and fills, for each stage, its name (static host string)
+ * and the time since the previous mark in milliseconds; returns the number of
+ * entries written (at most `cap`).  Off by default; not thread-safe.
+ */
+quads_status quads_moe_set_stage_trace(int32_t enable);
+int32_t quads_moe_get_stage_trace(const char** names /* host */, float* ms /* host */, int32_t cap);
+
 /* Number of kernels the last quads_* call on this host thread enqueued. */
 int32_t quads_last_launch_count(void);
 

@@ -254,3 +254,21 @@ def moe_last_kernel_ms():
     a, b = C.c_float(), C.c_float()
     check(lib.quads_moe_last_kernel_ms(C.byref(a), C.byref(b)))
     return a.value, b.value
+
+
+lib.quads_moe_set_stage_trace.restype = _i32
+lib.quads_moe_set_stage_trace.argtypes = [_i32]
+lib.quads_moe_get_stage_trace.restype = _i32
+lib.quads_moe_get_stage_trace.argtypes = [C.POINTER(C.c_char_p), C.POINTER(C.c_float), _i32]
+
+
+def moe_set_stage_trace(enable):
+    check(lib.quads_moe_set_stage_trace(1 if enable else 0))
+
+
+def moe_get_stage_trace():
+    """[(stage name, ms)] of the most recent traced MoE call."""
+    names = (C.c_char_p * 40)()
+    ms = (C.c_float * 40)()
+    n = lib.quads_moe_get_stage_trace(names, ms, 40)
+    return [(names[i].decode(), ms[i]) for i in range(n)]

@@ -71,9 +71,9 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // ------------------------------------------------------------------ workspace
 struct MoeLayout {
-  size_t header, amax, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
+  size_t header, amax, counters13, counters2, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
   size_t perm, pos_pad, row_token, row_weight;
-  size_t partials13, scores13, sel13, mask13, xq_pad, xsf, rq_pad, rsf;
+  size_t partials13, scores13, keys13, keys2, sel13, mask13, xq_pad, xsf, rq_pad, rsf;
   size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad;
   size_t total;
   int n_chunks, m_tiles_max, stats_ctas, rows_per_cta;
@@ -97,6 +97,8 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
   L.header = take(kHdrWords * 4);
   L.amax = take(16);
+  L.counters13 = take((size_t)((H + 31) / 32) * 4);
+  L.counters2 = take((size_t)((I + 31) / 32 + 1) * 4);
   L.ids = take((size_t)A * 4);
   L.wts = take((size_t)A * 4);
   L.chunk_counts = take((size_t)L.n_chunks * Ee * 4);
@@ -111,6 +113,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   L.row_weight = take(pad_rows * 4);
   L.partials13 = take((size_t)L.stats_ctas * H * 4);
   L.scores13 = take((size_t)H * 8 * kScoreSlices);
+  L.keys13 = take((size_t)H * 8);
   L.sel13 = take((size_t)H * 4);
   L.mask13 = take((size_t)H);
   L.xq_pad = take(pad_rows * (H / 2));
@@ -124,6 +127,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
     L.r2sf = take((size_t)L.m_tiles_max * (I / 64) * 512);
     L.partials2 = take((size_t)L.m_tiles_max * 4 * I * 4);
     L.scores2 = take((size_t)I * 8 * kScoreSlices);
+    L.keys2 = take((size_t)I * 8);
     L.sel2 = take((size_t)I * 4);
     L.mask2 = take((size_t)I);
     L.y_pad = take(pad_rows * (size_t)H * 2);
@@ -142,19 +146,36 @@ struct GemmTimers {
 };
 GemmTimers g_timers;
 
+// Optional stage trace of one MoE call: an event after every stage (off by default).
+struct StageTrace {
+  bool enabled = false;
+  int n = 0;
+  cudaEvent_t ev[40];
+  const char* name[40];
+  bool created = false;
+};
+StageTrace g_trace;
+inline void trace_mark(const char* name, cudaStream_t st) {
+  if (!g_trace.enabled || g_trace.n >= 40) return;
+  g_trace.name[g_trace.n] = name;
+  cudaEventRecord(g_trace.ev[g_trace.n], st);
+  ++g_trace.n;
+}
+
 int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
 
 quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
-                        int n_sel, double* slice_sums, uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
+                        int n_sel, double* slice_sums, unsigned int* counters, unsigned long long* keys,
+                        uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
   score_reduce_kernel<<<dim3((C + 31) / 32, kScoreSlices), 256, 0, st>>>(partials, n_part_ptr, n_part_mul,
-                                                                          n_part_fixed, C, slice_sums);
+                                                                          n_part_fixed, C, slice_sums, counters, keys);
   note_launch();
   static bool attr = false;
   if (!attr) {
     QUADS_CUDA_OK(cudaFuncSetAttribute(rank_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
     attr = true;
   }
-  rank_select_kernel<<<(C + 63) / 64, 256, (size_t)C * 8, st>>>(slice_sums, C, n_sel, mask);
+  rank_select_kernel<<<(C + 63) / 64, 256, (size_t)C * 8, st>>>(keys, C, n_sel, mask);
   note_launch();
   if (sel_export) {
     sel_list_kernel<<<1, 1024, 0, st>>>(mask, C, sel_export);
@@ -308,6 +329,27 @@ quads_status quads_moe_async_status(const void* workspace, void* cuda_stream) {
   return v == 0 ? QUADS_OK : (quads_status)v;
 }
 
+quads_status quads_moe_set_stage_trace(int32_t enable) {
+  if (enable && !g_trace.created) {
+    for (int i = 0; i < 40; ++i) QUADS_CUDA_OK(cudaEventCreate(&g_trace.ev[i]));
+    g_trace.created = true;
+  }
+  g_trace.enabled = enable != 0;
+  g_trace.n = 0;
+  return QUADS_OK;
+}
+
+int32_t quads_moe_get_stage_trace(const char** names, float* ms, int32_t cap) {
+  if (!names || !ms || g_trace.n < 2) return 0;
+  if (cudaEventSynchronize(g_trace.ev[g_trace.n - 1]) != cudaSuccess) return 0;
+  int n = 0;
+  for (int i = 1; i < g_trace.n && n < cap; ++i, ++n) {
+    names[n] = g_trace.name[i];
+    if (cudaEventElapsedTime(&ms[n], g_trace.ev[i - 1], g_trace.ev[i]) != cudaSuccess) return n;
+  }
+  return n;
+}
+
 quads_status quads_moe_set_kernel_timing(int32_t enable) {
   if (enable && !g_timers.created) {
     for (int i = 0; i < 4; ++i) QUADS_CUDA_OK(cudaEventCreate(&g_timers.ev[i]));
@@ -371,8 +413,11 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   const int A = T * topk;
   const size_t pad_rows = (size_t)L.m_tiles_max * 128;
 
+  g_trace.n = 0;
+  trace_mark("start", st);
   // header (status word included) and the amax word start at zero
   QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, L.ids, st));
+  trace_mark("memset", st);
 
   // ---- per-tensor scale of x
   if (!a->a13_gs) {
@@ -383,6 +428,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     note_launch();
   }
 
+  trace_mark("amax", st);
   // ---- routing and dispatch order
   if (dense) {
     dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, pos_pad, row_token, row_weight, tile_expert,
@@ -394,14 +440,17 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     route_kernel<<<L.n_chunks, 256, 0, st>>>(a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts,
                                               a->topk_ids, a->topk_w);
     note_launch();
+    trace_mark("route", st);
     scan_kernel<<<1, 1024, 0, st>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
                                    tile_rows, header, a->expert_offsets);
     note_launch();
+    trace_mark("scan", st);
     permute_kernel<<<(L.n_chunks + 3) / 4, 128, 0, st>>>(T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm,
                                                pos_pad, row_token, row_weight, a->perm);
     note_launch();
   }
 
+  trace_mark("permute", st);
   // ---- site 13: statistics, selection, quantize + residual + dispatch scatter
   const int nsel13 = a->rac_nsel_13;
   float* gs13_store = a->a13_gs_out;
@@ -412,12 +461,14 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
         a->xq, a->xsf);
     note_launch();
   }
+  trace_mark("rac_stats", st);
   if (nsel13 > 0) {
     s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
-                   reinterpret_cast<double*>(P(L.scores13)), mask13, a->sel13, st);
+                   reinterpret_cast<double*>(P(L.scores13)), reinterpret_cast<unsigned int*>(P(L.counters13)),
+                   reinterpret_cast<unsigned long long*>(P(L.keys13)), mask13, a->sel13, st);
     if (s != QUADS_OK) return s;
   }
-  // the dispatch kernel needs the scale as a value in memory: the amax word or the caller's
+  trace_mark("select13", st);
   {
     const int64_t groups = (int64_t)T * (H / 64);
     rac_dispatch_kernel<<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(
@@ -426,6 +477,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     note_launch();
   }
 
+  trace_mark("rac_dispatch", st);
   // ---- tensor maps
   CUtensorMap tm_x, tm_r, tm_w13;
   if ((s = make_codes_map(&tm_x, P(L.xq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
@@ -463,12 +515,14 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   if ((s = launch_gemm(kEpiSwiGLU, g, tm_x, tm_r, tm_w13, di.sm_count, st)) != QUADS_OK) return s;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[1], st));
 
+  trace_mark("gemm1", st);
   // ---- site 2: selection and masking of the residual of h
   const int nsel2 = a->rac_nsel_2;
   uint8_t* mask2 = P(L.mask2);
   if (nsel2 > 0) {
     s = run_select(g.partials2, header + kHdrMTiles, 4 /* one partial row per tile and lane quadrant */, 0, I, nsel2,
-                   reinterpret_cast<double*>(P(L.scores2)), mask2, a->sel2, st);
+                   reinterpret_cast<double*>(P(L.scores2)), reinterpret_cast<unsigned int*>(P(L.counters2)),
+                   reinterpret_cast<unsigned long long*>(P(L.keys2)), mask2, a->sel2, st);
     if (s != QUADS_OK) return s;
     mask_codes_kernel<<<di.sm_count * 8, 256, 0, st>>>(P(L.r2q_pad), header + kHdrPaddedRows, I, mask2);
     note_launch();
@@ -483,6 +537,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     note_launch();
   }
 
+  trace_mark("select2+mask", st);
   // ---- second projection + weighted combine
   uint16_t* y_pad = reinterpret_cast<uint16_t*>(P(L.y_pad));
   CUtensorMap tm_h, tm_r2, tm_w2;
@@ -506,10 +561,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
     g_timers.valid = true;
   }
+  trace_mark("gemm2", st);
   const int64_t n8 = (int64_t)T * (H / 8);
   combine_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(y_pad, pos_pad, wts, T, H, topk,
                                                                 static_cast<uint16_t*>(a->out));
   note_launch();
+  trace_mark("combine", st);
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
 }

@@ -56,23 +56,22 @@ __device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
 }
 
 // Two floats -> one byte of E2M1 codes (lo in bits 0..3, hi in bits 4..7),
-// round-to-nearest-even, saturating to 6.  The sign bit is forced to the sign
-// of the input so that values rounding to zero keep it.
+// round-to-nearest-even, saturating to 6.  The hardware convert keeps the sign
+// bit of values that round to zero (-0, small negatives), which is the
+// convention of this library; the exhaustive quantizer test pins it.
 __device__ __forceinline__ uint32_t f32x2_to_e2m1x2(float lo, float hi) {
   uint16_t r;
   asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; cvt.u16.u8 %0, t; }"
       : "=h"(r) : "f"(hi), "f"(lo));
-  uint32_t s = ((__float_as_uint(lo) >> 31) << 3) | ((__float_as_uint(hi) >> 31) << 7);
-  return ((uint32_t)r & 0x77u) | s;
+  return (uint32_t)r & 0xFFu;
 }
 
-// E2M1 nibble -> float (exact): 0, .5, 1, 1.5, 2, 3, 4, 6 with sign in bit 3.
-__device__ __forceinline__ float e2m1_to_f32(uint32_t c) {
-  uint32_t m = c & 7u;
-  // magnitudes in halves: 0,1,2,3,4,6,8,12
-  uint32_t halves = (m < 2u) ? m : ((2u | (m & 1u)) << ((m >> 1) - 1u));
-  float v = 0.5f * (float)halves;
-  return (c & 8u) ? -v : v;
+// One byte of two E2M1 codes -> two floats (exact): low nibble -> .x, high nibble -> .y.
+__device__ __forceinline__ float2 e2m1x2_to_f32x2(uint32_t byte) {
+  uint32_t h2;
+  uint16_t in = (uint16_t)(byte & 0xFFu);
+  asm("{ .reg .b8 t; cvt.u8.u16 t, %1; cvt.rn.f16x2.e2m1x2 %0, t; }" : "=r"(h2) : "h"(in));
+  return __half22float2(*reinterpret_cast<__half2*>(&h2));
 }
 
 struct BlockQ {
@@ -107,9 +106,13 @@ __device__ __forceinline__ BlockQ quantize_block(const float* v, float gs) {
 // Dequantize the 16 codes of a block: value(code) * d, one float32 multiply.
 __device__ __forceinline__ void dequant_block(const BlockQ& q, float* out) {
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    out[i] = __fmul_rn(e2m1_to_f32((q.lo >> (4 * i)) & 0xFu), q.d);
-    out[8 + i] = __fmul_rn(e2m1_to_f32((q.hi >> (4 * i)) & 0xFu), q.d);
+  for (int i = 0; i < 4; ++i) {
+    const float2 a = e2m1x2_to_f32x2(q.lo >> (8 * i));
+    const float2 b = e2m1x2_to_f32x2(q.hi >> (8 * i));
+    out[2 * i] = __fmul_rn(a.x, q.d);
+    out[2 * i + 1] = __fmul_rn(a.y, q.d);
+    out[8 + 2 * i] = __fmul_rn(b.x, q.d);
+    out[9 + 2 * i] = __fmul_rn(b.y, q.d);
   }
 }
 

@@ -11,14 +11,15 @@
 // accumulator in tensor memory, which is possible because the residual shares
 // the per-tensor scale of its activation.
 //
-// One persistent CTA per SM, 10 warps:
+// One persistent CTA per SM, 18 warps:
 //   warp 0     producer: TMA tile loads of packed FP4 (128-byte swizzle) and bulk
 //              copies of 512-byte scale atoms into a 3-stage shared-memory ring;
 //   warp 1     tensor-memory allocation; one thread copies scale atoms to TMEM
 //              (tcgen05.cp) and issues the MMAs, releasing stages with
 //              tcgen05.commit;
-//   warps 2..9 epilogue: drain the 128 x 256 accumulator into registers, free it
-//              for the next tile at once, then run the fused epilogue.
+//   warps 2..17 epilogue: drain the 128 x 256 accumulator into registers (64
+//              columns per thread), free it for the next tile at once, then run
+//              the fused epilogue.  Four warps per scheduler hide its latencies.
 // Tile = 128 dispatch rows x 256 weight rows; K is consumed 256 elements per
 // stage (four K=64 MMAs).  Every wait is bounded; a wait that gives up records
 // QUADS_ERR_TIMEOUT in the status word and all roles leave.
@@ -44,7 +45,8 @@ constexpr int kOffSfB = kOffSfR + kSfA;
 constexpr int kStageBytes = kOffSfB + kSfB;       // 73728
 constexpr int kBarOffset = kStages * kStageBytes; // barriers after the ring
 constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // + barrier block + alignment slack
-constexpr int kThreads = 320;
+constexpr int kThreads = 576;
+constexpr int kEpiWarps = 16;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256;                  // accumulator: columns 0..255
 constexpr int kTmemSfPerBuf = 64;                 // SFA 16 | SFR 16 | SFB 32, double buffered
@@ -228,7 +230,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
       mbar_init(bar_empty + 8 * s, 1);
     }
     mbar_init(bar_tfull, 1);
-    mbar_init(bar_tempty, 8);
+    mbar_init(bar_tempty, kEpiWarps);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tmap(&tm_a);
@@ -329,7 +331,7 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
   } else {
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;                 // TMEM lane quadrant this warp may access
-    const int hf = (warp - 2) >> 2;         // which half of the tile's columns
+    const int cq = (warp - 2) >> 2;         // which quarter of the tile's columns (0..3)
     const int row_in_tile = q * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const float a_gs = p.a_gs ? p.a_gs[0]
@@ -346,16 +348,14 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
       ok = mbar_wait(bar_tfull, (uint32_t)(it & 1), abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
-      float acc[128];
+      float acc[64];
       if (EPI == kEpiSwiGLU) {
-        // gate columns [hf*64, +64) -> acc[0..63]; up columns [128 + hf*64, +64) -> acc[64..127]
-        tmem_ld32(lane_addr + hf * 64, acc);
-        tmem_ld32(lane_addr + hf * 64 + 32, acc + 32);
-        tmem_ld32(lane_addr + 128 + hf * 64, acc + 64);
-        tmem_ld32(lane_addr + 128 + hf * 64 + 32, acc + 96);
+        // gate columns [cq*32, +32) -> acc[0..31]; up columns [128 + cq*32, +32) -> acc[32..63]
+        tmem_ld32(lane_addr + cq * 32, acc);
+        tmem_ld32(lane_addr + 128 + cq * 32, acc + 32);
       } else {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(lane_addr + hf * 128 + 32 * c, acc + 32 * c);
+        tmem_ld32(lane_addr + cq * 64, acc);
+        tmem_ld32(lane_addr + cq * 64 + 32, acc + 32);
       }
       tmem_ld_wait();
       tc_fence_before();
@@ -365,18 +365,18 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
       if (EPI == kEpiSwiGLU) {
         const float h_gs = p.h_gs[0];
         const int I = p.n_out;
-        const int f0 = nt * 128 + hf * 64;        // first feature of this thread's 64
+        const int f0 = nt * 128 + cq * 32;        // first feature of this thread's 32
         const int kt2 = I >> 6;
         uint32_t hs = 0, rs = 0;
         int drow = 0;
         if (p.h_export) drow = p.offsets[e] + (mt - p.tile_prefix[e]) * kBM + row_in_tile;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
           float hb[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float g = __fmul_rn(acc[16 * c + i], scale);
-            const float u = __fmul_rn(acc[64 + 16 * c + i], scale);
+            const float u = __fmul_rn(acc[32 + 16 * c + i], scale);
             const float h = __fdividef(g, 1.0f + __expf(-g)) * u;
             hb[i] = __bfloat162float(__float2bfloat16_rn(h));
           }
@@ -413,18 +413,19 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
           }
         }
         if (valid) {
+          // this thread's two scale bytes: blocks (f0/16) and (f0/16)+1, adjacent in the atom
           const size_t so = sf_tiled_offset(prow, f0 >> 4, kt2);
-          *reinterpret_cast<uint32_t*>(p.hsf_tiled + so) = hs;
-          if (p.resid2) *reinterpret_cast<uint32_t*>(p.r2sf_tiled + so) = rs;
+          *reinterpret_cast<uint16_t*>(p.hsf_tiled + so) = (uint16_t)hs;
+          if (p.resid2) *reinterpret_cast<uint16_t*>(p.r2sf_tiled + so) = (uint16_t)rs;
         }
       } else if (EPI == kEpiCombine) {
         // y = W2 h~ for this dispatched row, rounded to bf16; the weighted sum over a
         // token's experts is taken afterwards in a fixed order (no atomics).
-        const int n0 = nt * 256 + hf * 128;
+        const int n0 = nt * 256 + cq * 64;
         if (valid && n0 < p.n_out) {
           uint16_t* dst = p.y_pad + (size_t)prow * p.n_out + n0;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < 4; ++i)
             stg256(dst + 16 * i,
                    f32x2_to_bf16x2(acc[16 * i] * scale, acc[16 * i + 1] * scale),
                    f32x2_to_bf16x2(acc[16 * i + 2] * scale, acc[16 * i + 3] * scale),
@@ -436,11 +437,11 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
                    f32x2_to_bf16x2(acc[16 * i + 14] * scale, acc[16 * i + 15] * scale));
         }
       } else {
-        const int n0 = nt * 256 + hf * 128;
+        const int n0 = nt * 256 + cq * 64;
         if (valid && n0 < p.n_out) {
           uint4* dst = reinterpret_cast<uint4*>(p.out_bf16 + (size_t)p.row_token[prow] * p.n_out + n0);
 #pragma unroll
-          for (int i = 0; i < 16; ++i)
+          for (int i = 0; i < 8; ++i)
             dst[i] = make_uint4(f32x2_to_bf16x2(acc[8 * i] * scale, acc[8 * i + 1] * scale),
                                 f32x2_to_bf16x2(acc[8 * i + 2] * scale, acc[8 * i + 3] * scale),
                                 f32x2_to_bf16x2(acc[8 * i + 4] * scale, acc[8 * i + 5] * scale),

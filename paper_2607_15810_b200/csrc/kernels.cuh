@@ -24,8 +24,9 @@ __global__ void rac_stats_kernel(const uint16_t* x, int T, int H, const float* g
                                  uint8_t* xsf_out);
 constexpr int kScoreSlices = 16;
 __global__ void score_reduce_kernel(const float* partials, const int* n_part_ptr, int n_part_mul,
-                                    int n_part_fixed, int C, double* slice_sums);
-__global__ void rank_select_kernel(const double* slice_sums, int C, int n_sel, uint8_t* mask);
+                                    int n_part_fixed, int C, double* slice_sums, unsigned int* counters,
+                                    unsigned long long* score_keys);
+__global__ void rank_select_kernel(const unsigned long long* score_keys, int C, int n_sel, uint8_t* mask);
 __global__ void sel_list_kernel(const uint8_t* mask, int C, int32_t* sel_export);
 __global__ void rac_dispatch_kernel(const uint16_t* x, int T, int H, const float* gs_in,
                                     const uint32_t* amax_bits, int n_sel,

@@ -154,13 +154,17 @@ rac_stats_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
   }
 }
 
-// Channel scores, stage 1: the partial rows are split into kScoreSlices
-// contiguous slices; CTA (column group, slice) adds its slice's rows in a fixed
-// order in float64.  grid = (ceil(C/32), kScoreSlices), 256 threads = 32 columns
-// x 8 interleaved row lanes.
+// Channel scores (Eq. channel-score).  The partial rows are split into
+// kScoreSlices contiguous slices; CTA (column group, slice) adds its slice's
+// rows in float64.  The CTA of a column group that finishes last adds the
+// slice sums in slice order (a fixed order, whichever CTA does it) and stores
+// the group's 32 scores as order-preserving 64-bit keys (scores are >= 0).
+// grid = (ceil(C/32), kScoreSlices), 256 threads = 32 columns x 8 row lanes.
+// `counters` (one per column group) must be zero on entry.
 __global__ void __launch_bounds__(256)
 score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ n_part_ptr, int n_part_mul,
-                    int n_part_fixed, int C, double* __restrict__ slice_sums) {
+                    int n_part_fixed, int C, double* __restrict__ slice_sums, unsigned int* __restrict__ counters,
+                    unsigned long long* __restrict__ score_keys) {
   const int n_part = n_part_ptr ? *n_part_ptr * n_part_mul : n_part_fixed;
   const int per = (n_part + kScoreSlices - 1) / kScoreSlices;
   const int p0 = blockIdx.y * per, p1 = min(n_part, p0 + per);
@@ -170,6 +174,7 @@ score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ 
   if (col < C)
     for (int p = p0 + rl; p < p1; p += 8) s += (double)partials[(size_t)p * C + col];
   __shared__ double sm[8][32];
+  __shared__ unsigned int last;
   sm[rl][threadIdx.x & 31] = s;
   __syncthreads();
   if (rl == 0 && col < C) {
@@ -178,31 +183,38 @@ score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ 
     for (int i = 0; i < 8; ++i) t += sm[i][threadIdx.x & 31];
     slice_sums[(size_t)blockIdx.y * C + col] = t;
   }
-}
-
-// Channel selection (Eq. channel-select), stage 2: every CTA rebuilds all C
-// scores (slice sums added in slice order) in shared memory, then ranks 64
-// channels: rank_j = #{i : s_i > s_j, or s_i == s_j and i < j}; channel j is
-// selected iff rank_j < n_sel (the n_sel largest, ties to the lower index).
-// grid = ceil(C/64), 256 threads (4 per ranked channel), smem = C doubles.
-__global__ void __launch_bounds__(256)
-rank_select_kernel(const double* __restrict__ slice_sums, int C, int n_sel, uint8_t* __restrict__ mask) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* sc = reinterpret_cast<double*>(smem_raw);
-  for (int i = threadIdx.x; i < C; i += blockDim.x) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = atomicAdd(counters + blockIdx.x, 1u);
+  __syncthreads();
+  if (last == kScoreSlices - 1 && rl == 0 && col < C) {
+    __threadfence();
     double t = 0.0;
 #pragma unroll
-    for (int s = 0; s < kScoreSlices; ++s) t += slice_sums[(size_t)s * C + i];
-    sc[i] = t;
+    for (int i = 0; i < kScoreSlices; ++i) t += __ldcg(slice_sums + (size_t)i * C + col);
+    score_keys[col] = (unsigned long long)__double_as_longlong(t);
   }
+}
+
+// Channel selection (Eq. channel-select): rank_j = #{i : s_i > s_j, or s_i ==
+// s_j and i < j}; channel j is selected iff rank_j < n_sel (the n_sel largest,
+// ties to the lower index).  Every CTA loads all C score keys into shared
+// memory and ranks 64 channels with 4 threads each.
+// grid = ceil(C/64), 256 threads, smem = C * 8 bytes.
+__global__ void __launch_bounds__(256)
+rank_select_kernel(const unsigned long long* __restrict__ score_keys, int C, int n_sel, uint8_t* __restrict__ mask) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* sc = reinterpret_cast<unsigned long long*>(smem_raw);
+  for (int i = threadIdx.x; i < C; i += blockDim.x) sc[i] = score_keys[i];
   __syncthreads();
   const int j = blockIdx.x * 64 + (threadIdx.x >> 2);
   const int sub = threadIdx.x & 3;
   int rank = 0;
   if (j < C) {
-    const double sj = sc[j];
+    const unsigned long long sj = sc[j];
+#pragma unroll 8
     for (int i = sub; i < C; i += 4) {
-      const double si = sc[i];
+      const unsigned long long si = sc[i];
       rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
     }
   }

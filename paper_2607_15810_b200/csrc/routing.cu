@@ -5,10 +5,18 @@
 
 namespace quads {
 
-// One warp per token.  E <= 256.  Top-k by logit, ties to the lower expert id,
-// slots in descending-logit order; weights = softmax over all experts at the
-// chosen ones, optionally renormalised.  Each CTA (kRouteTokensPerCta tokens)
-// also writes its per-expert assignment counts: chunk_counts[cta][E].
+// Order-preserving map float -> uint32 (larger float <=> larger uint).
+__device__ __forceinline__ uint32_t float_key(float v) {
+  const uint32_t b = __float_as_uint(v);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Each warp routes kRouteTokensPerWarp tokens at once (independent chains hide
+// the reduction latency).  E <= 256.  Top-k by logit, ties to the lower expert
+// id, slots in descending-logit order; weights = softmax over all experts at
+// the chosen ones, optionally renormalised.  Each CTA (kRouteTokensPerCta
+// tokens) also writes its per-expert assignment counts: chunk_counts[expert][cta].
+constexpr int kRouteTokensPerWarp = 4;
 __global__ void __launch_bounds__(256)
 route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
              int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
@@ -17,61 +25,90 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
   for (int i = threadIdx.x; i < E; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t0 = blockIdx.x * kRouteTokensPerCta;
-  for (int tt = warp; tt < kRouteTokensPerCta; tt += (int)(blockDim.x >> 5)) {
-    const int t = t0 + tt;
-    if (t >= T) break;
-    float v[8];
+  const int t0 = blockIdx.x * kRouteTokensPerCta + warp * kRouteTokensPerWarp;
+  constexpr int TW = kRouteTokensPerWarp;
+  float v[TW][8];
+  float mx[TW], sum[TW], wsum[TW], my_w[TW];
+  int my_id[TW];
+#pragma unroll
+  for (int a = 0; a < TW; ++a) {
+    const int t = t0 + a;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int e = j * 32 + lane;
-      v[j] = e < E ? logits[(size_t)t * E + e] : -INFINITY;
+      v[a][j] = (t < T && e < E) ? logits[(size_t)t * E + e] : -INFINITY;
     }
-    // softmax denominator over all experts
-    float mx = v[0];
+  }
 #pragma unroll
-    for (int j = 1; j < 8; ++j) mx = fmaxf(mx, v[j]);
-    mx = warp_max(mx);
-    float sum = 0.f;
+  for (int a = 0; a < TW; ++a) {
+    float m = v[a][0];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) sum += (j * 32 + lane < E) ? expf(v[j] - mx) : 0.f;
+    for (int j = 1; j < 8; ++j) m = fmaxf(m, v[a][j]);
+    mx[a] = m;
+  }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-    float my_w = 0.f;      // lane s keeps slot s
-    int my_id = -1;
-    float wsum = 0.f;
-    for (int s = 0; s < topk; ++s) {
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int a = 0; a < TW; ++a) mx[a] = fmaxf(mx[a], __shfl_xor_sync(0xFFFFFFFFu, mx[a], o));
+#pragma unroll
+  for (int a = 0; a < TW; ++a) {
+    float sacc = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sacc += (j * 32 + lane < E && t0 + a < T) ? expf(v[a][j] - mx[a]) : 0.f;
+    sum[a] = sacc; wsum[a] = 0.f; my_w[a] = 0.f; my_id[a] = 0;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int a = 0; a < TW; ++a) sum[a] += __shfl_xor_sync(0xFFFFFFFFu, sum[a], o);
+  for (int s = 0; s < topk; ++s) {
+    uint32_t bk[TW];
+    int be[TW];
+#pragma unroll
+    for (int a = 0; a < TW; ++a) {
       float bv = -INFINITY;
-      int be = 0x7FFFFFFF;
+      int e1 = 0x7FFFFFFF;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int e = j * 32 + lane;
-        if (e < E && (v[j] > bv)) { bv = v[j]; be = e; }    // ascending e within a lane: first max wins
+        if (e < E && v[a][j] > bv) { bv = v[a][j]; e1 = e; }   // ascending e: the first maximum wins
       }
+      bk[a] = (e1 == 0x7FFFFFFF) ? 0u : float_key(bv);
+      be[a] = e1;
+    }
+    uint32_t gk[TW];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
-        const int oe = __shfl_xor_sync(0xFFFFFFFFu, be, o);
-        if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
-      }
-      const float w = expf(bv - mx) / sum;
-      wsum += w;
-      if (lane == s) { my_w = w; my_id = be; }
+    for (int a = 0; a < TW; ++a) gk[a] = __reduce_max_sync(0xFFFFFFFFu, bk[a]);
+#pragma unroll
+    for (int a = 0; a < TW; ++a)
+      be[a] = (int)__reduce_min_sync(0xFFFFFFFFu, (unsigned)((bk[a] == gk[a]) ? be[a] : 0x7FFFFFFF));
+#pragma unroll
+    for (int a = 0; a < TW; ++a) {
+      // the winner's logit: recover from the key
+      const uint32_t kb = gk[a];
+      const float bv = __uint_as_float((kb & 0x80000000u) ? (kb & 0x7FFFFFFFu) : ~kb);
+      const float w = expf(bv - mx[a]) / sum[a];
+      wsum[a] += w;
+      if (lane == s) { my_w[a] = w; my_id[a] = be[a]; }
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        if (j * 32 + lane == be) v[j] = -INFINITY;         // remove the winner
+        if (j * 32 + lane == be[a]) v[a][j] = -INFINITY;       // remove the winner
     }
-    if (lane < topk) {
-      if (renormalize) my_w = my_w / wsum;
-      ids[(size_t)t * topk + lane] = my_id;
-      wts[(size_t)t * topk + lane] = my_w;
-      if (ids_out) ids_out[(size_t)t * topk + lane] = my_id;
-      if (wts_out) wts_out[(size_t)t * topk + lane] = my_w;
-      atomicAdd(&hist[my_id], 1);
+  }
+#pragma unroll
+  for (int a = 0; a < TW; ++a) {
+    const int t = t0 + a;
+    if (t < T && lane < topk) {
+      const float w = renormalize ? my_w[a] / wsum[a] : my_w[a];
+      ids[(size_t)t * topk + lane] = my_id[a];
+      wts[(size_t)t * topk + lane] = w;
+      if (ids_out) ids_out[(size_t)t * topk + lane] = my_id[a];
+      if (wts_out) wts_out[(size_t)t * topk + lane] = w;
+      atomicAdd(&hist[my_id[a]], 1);
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < E; i += blockDim.x) chunk_counts[(size_t)blockIdx.x * E + i] = hist[i];
+  for (int i = threadIdx.x; i < E; i += blockDim.x) chunk_counts[(size_t)i * gridDim.x + blockIdx.x] = hist[i];
 }
 
 // One CTA of 1024 threads.  A warp per expert (round robin): exclusive prefix of
@@ -88,17 +125,25 @@ scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
   for (int e = warp; e < E; e += n_warps) {
     int run = 0;
-    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
-      const int c = c0 + lane;
-      const int v = c < n_chunks ? chunk_counts[(size_t)c * E + e] : 0;
-      int incl = v;
+    for (int c0 = 0; c0 < n_chunks; c0 += 256) {
+      int v[8];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += n;
+      for (int k = 0; k < 8; ++k) {              // all loads first: one memory latency per 256 chunks
+        const int c = c0 + k * 32 + lane;
+        v[k] = c < n_chunks ? chunk_counts[(size_t)e * n_chunks + c] : 0;
       }
-      if (c < n_chunks) chunk_base[(size_t)c * E + e] = run + incl - v;
-      run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int c = c0 + k * 32 + lane;
+        int incl = v[k];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += n;
+        }
+        if (c < n_chunks) chunk_base[(size_t)e * n_chunks + c] = run + incl - v[k];
+        run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      }
     }
     if (lane == 0) cnt[e] = run;
   }
@@ -142,7 +187,7 @@ permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = blockIdx.x * 4 + warp;
   if (chunk >= n_chunks) return;
-  for (int e = lane; e < E; e += 32) run[warp][e] = chunk_base[(size_t)chunk * E + e];
+  for (int e = lane; e < E; e += 32) run[warp][e] = chunk_base[(size_t)e * n_chunks + chunk];
   __syncwarp();
   const int t0 = chunk * kRouteTokensPerCta;
   const int n = min(kRouteTokensPerCta, T - t0) * topk;

@@ -1,5 +1,6 @@
 // C ABI entry points: argument checks, workspace carving, TMA descriptors and
 // the launch sequence of each public call.
+#include <cstdlib>
 #include <mutex>
 
 #include "kernels.cuh"
@@ -59,10 +60,12 @@ quads_status make_codes_map(CUtensorMap* map, const void* base, uint64_t rows, u
   if (rows == 0) rows = 1;
   cuuint64_t dims[2] = {row_bytes, rows};
   cuuint64_t strides[1] = {row_bytes};
-  cuuint32_t box[2] = {128, 128};
+  cuuint32_t box[2] = {(cuuint32_t)kGemmStageKBytes, 128};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  kGemmStageKBytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? QUADS_OK : QUADS_ERR_CUDA;
 }
@@ -85,7 +88,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   const int64_t A = dense ? T : (int64_t)T * topk;
   const int Ee = dense ? 1 : E;
   L.n_chunks = (T + kRouteTokensPerCta - 1) / kRouteTokensPerCta;
-  L.m_tiles_max = (int)(A / 128) + Ee;
+  L.m_tiles_max = ((int)(A / (128 * kMTileGroup)) + Ee) * kMTileGroup;
   L.stats_ctas = T < 592 * 4 ? (T + 3) / 4 : 592;
   if (L.stats_ctas < 1) L.stats_ctas = 1;
   L.rows_per_cta = (T + L.stats_ctas - 1) / L.stats_ctas;
@@ -162,7 +165,15 @@ inline void trace_mark(const char* name, cudaStream_t st) {
   ++g_trace.n;
 }
 
-int pow2_at_least(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+// 1: single-CTA tiles of 128 x 256 (default, the faster one as measured); 2: CTA pairs computing
+// 256 x 256 tiles with cta_group::2 MMAs, selected with QUADS_GEMM_CTA_GROUP=2.
+int gemm_cta_group() {
+  static int v = [] {
+    const char* e = getenv("QUADS_GEMM_CTA_GROUP");
+    return (e && e[0] == '2') ? 2 : 1;
+  }();
+  return v;
+}
 
 quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
                         int n_sel, double* slice_sums, unsigned int* counters, unsigned long long* keys,
@@ -494,13 +505,14 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.row_token = row_token; g.row_weight = row_weight;
   g.tile_prefix = tile_prefix; g.offsets = offsets;
   g.status = header + kHdrStatus;
+  { const char* e = getenv("QUADS_DBG"); g.dbg = e ? atoi(e) : 0; }
   g.b_rows_per_expert = N1;
   if (dense) {
     g.n_out = a->N;
     g.n_tiles_n = (a->N + 255) / 256;
     g.half1_row_offset = 128;
     g.out_bf16 = static_cast<uint16_t*>(a->out);
-    return launch_gemm(kEpiStore, g, tm_x, tm_r, tm_w13, di.sm_count, st);
+    return launch_gemm(kEpiStore, gemm_cta_group(), g, tm_x, tm_r, tm_w13, di.sm_count, st);
   }
   g.n_out = I;
   g.n_tiles_n = I / 128;
@@ -512,7 +524,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.h_export = static_cast<uint16_t*>(a->h_bf16);
   const bool timing = g_timers.enabled && g_timers.created;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[0], st));
-  if ((s = launch_gemm(kEpiSwiGLU, g, tm_x, tm_r, tm_w13, di.sm_count, st)) != QUADS_OK) return s;
+  if ((s = launch_gemm(kEpiSwiGLU, gemm_cta_group(), g, tm_x, tm_r, tm_w13, di.sm_count, st)) != QUADS_OK) return s;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[1], st));
 
   trace_mark("gemm1", st);
@@ -556,7 +568,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g2.half1_row_offset = 128;
   g2.y_pad = y_pad;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[2], st));
-  if ((s = launch_gemm(kEpiCombine, g2, tm_h, tm_r2, tm_w2, di.sm_count, st)) != QUADS_OK) return s;
+  if ((s = launch_gemm(kEpiCombine, gemm_cta_group(), g2, tm_h, tm_r2, tm_w2, di.sm_count, st)) != QUADS_OK) return s;
   if (timing) {
     QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
     g_timers.valid = true;

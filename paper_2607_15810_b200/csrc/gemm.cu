@@ -11,6 +11,13 @@
 // accumulator in tensor memory, which is possible because the residual shares
 // the per-tensor scale of its activation.
 //
+// Two variants share the code: CG = 1 (one CTA per tile of 128 x 256) and CG = 2
+// (a cluster of two CTAs computes a 256 x 256 tile with `cta_group::2` MMAs:
+// each CTA holds its own 128 rows of A^ / R^ and HALF of the weight tile, so the
+// bytes every SM must pull from L2 per flop drop by about a quarter -- the
+// single-CTA kernel is bound by exactly that ingest, not by the tensor pipe).
+// No TMA multicast is used: every CTA loads what it needs itself.
+//
 // One persistent CTA per SM, 18 warps:
 //   warp 0     producer: TMA tile loads of packed FP4 (128-byte swizzle) and bulk
 //              copies of 512-byte scale atoms into a 3-stage shared-memory ring;
@@ -31,25 +38,30 @@ namespace {
 
 constexpr int kBM = 128;
 constexpr int kBN = 256;
-constexpr int kStageKBytes = 128;                 // 256 FP4 elements per row per stage
-constexpr int kStages = 3;
-constexpr int kTileA = kBM * kStageKBytes;        // 16384
-constexpr int kTileB = kBN * kStageKBytes;        // 32768
-constexpr int kSfA = 4 * 512;                     // 4 atoms (128 rows x 4 blocks each)
-constexpr int kSfB = 2 * kSfA;
+constexpr int kKSteps = kGemmKSteps;              // K = 64 MMAs per pipeline stage
+constexpr int kStageKBytes = kGemmStageKBytes;    // bytes of packed FP4 per row per stage
+constexpr int kTileA = kBM * kStageKBytes;
+constexpr int kSfA = kKSteps * 512;               // one atom (128 rows x 4 blocks) per K step
+constexpr int kSfB = 2 * kSfA;                    // scales of all 256 weight rows
 constexpr int kOffR = kTileA;
 constexpr int kOffB = 2 * kTileA;
-constexpr int kOffSfA = kOffB + kTileB;
-constexpr int kOffSfR = kOffSfA + kSfA;
-constexpr int kOffSfB = kOffSfR + kSfA;
-constexpr int kStageBytes = kOffSfB + kSfB;       // 73728
-constexpr int kBarOffset = kStages * kStageBytes; // barriers after the ring
-constexpr int kSmemBytes = kBarOffset + 256 + 1024;  // + barrier block + alignment slack
 constexpr int kThreads = 576;
 constexpr int kEpiWarps = 16;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256;                  // accumulator: columns 0..255
-constexpr int kTmemSfPerBuf = 64;                 // SFA 16 | SFR 16 | SFB 32, double buffered
+constexpr int kTmemSfPerBuf = 16 * kKSteps;       // SFA 4/step | SFR 4/step | SFB 8/step, double buffered
+
+template <int CG>
+struct Cfg {
+  static constexpr int kTileB = kBN * kStageKBytes / CG;     // weight rows held by one CTA
+  static constexpr int kStages = (CG == 1 ? 12 : 16) / kKSteps;   // ~216 KB of ring either way
+  static constexpr int kOffSfA = kOffB + kTileB;
+  static constexpr int kOffSfR = kOffSfA + kSfA;
+  static constexpr int kOffSfB = kOffSfR + kSfA;
+  static constexpr int kStageBytes = kOffSfB + kSfB;         // 73728 / 57344
+  static constexpr int kBarOffset = kStages * kStageBytes;   // barriers after the ring
+  static constexpr int kSmemBytes = kBarOffset + 256 + 1024; // + barrier block + alignment slack
+};
 constexpr uint64_t kWaitNs = 2000000000ull;       // bound of every device-side wait (2 s)
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -104,6 +116,13 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// L2 prefetches: warm the cache for a later stage without needing a free shared-memory slot.
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_prefetch(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -111,25 +130,107 @@ __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+template <int CG>
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (CG == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  } else {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
 }
+template <int CG>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+  if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+  else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
+// Arrive on `bar` once all tcgen05 operations issued so far by this thread are
+// complete.  CG == 2: the arrival is delivered to the barrier at the same
+// shared-memory offset in both CTAs of the pair.
+template <int CG>
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  if (CG == 1) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  } else {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+  }
 }
+template <int CG>
 __device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+  if (CG == 1) asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+  else asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
+template <int CG>
 __device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %6, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate) : "memory");
+  if (CG == 1) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate) : "memory");
+  }
+}
+
+// True in exactly one lane of a fully active warp.  The single-thread tcgen05 /
+// TMA instructions are issued under this predicate from warp-uniform code, so
+// that their operands are computed once per warp (uniform datapath) instead of
+// being moved lane-by-lane inside a divergent branch.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
+// ---- cluster helpers (CG == 2)
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait on a barrier that also receives arrivals from the peer CTA.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  int32_t* status) {
+  if (mbar_try_cluster(bar, parity)) return true;
+  const uint64_t t0 = globaltimer();
+  uint32_t spins = 0;
+  while (!mbar_try_cluster(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > kWaitNs) {
+        *abort_flag = 1;
+        atomicExch(status, (int32_t)QUADS_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
 }
 
 // 32 consecutive accumulator columns of this thread's TMEM lane.
@@ -161,8 +262,11 @@ __device__ __forceinline__ uint64_t desc_sf_atom(uint32_t saddr) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
 }
 // Instruction descriptor: E2M1 x E2M1, UE4M3 block scales, both operands
-// K-major, M = 128, N = 256, dense.
-constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+// K-major, M = 128 per CTA of the group, N = 256, dense.
+template <int CG>
+__host__ __device__ constexpr uint32_t idesc_nvf4() {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)((kBM * CG) >> 4) << 24);
+}
 
 __device__ __forceinline__ void stg256(void* addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
                                        uint32_t f, uint32_t g, uint32_t h) {
@@ -171,8 +275,8 @@ __device__ __forceinline__ void stg256(void* addr, uint32_t a, uint32_t b, uint3
 }
 
 struct __align__(8) BarrierBlock {
-  uint64_t full[kStages];
-  uint64_t empty[kStages];
+  uint64_t full[8];
+  uint64_t empty[8];
   uint64_t tmem_full;
   uint64_t tmem_empty;
   uint32_t tmem_base;
@@ -209,14 +313,15 @@ __device__ __forceinline__ float warp_colsum16(const float* v, int lane) {
   return d;
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_r,
-            const __grid_constant__ CUtensorMap tm_b) {
+template <int EPI, int CG>
+__device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap* tm_a, const CUtensorMap* tm_r,
+                                          const CUtensorMap* tm_b) {
+  using C = Cfg<CG>;
+  constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_dyn[];
   const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_dyn + (smem_base - smem_u32(smem_dyn));
-  BarrierBlock* bars = reinterpret_cast<BarrierBlock*>(smem_gen + kBarOffset);
+  BarrierBlock* bars = reinterpret_cast<BarrierBlock*>(smem_gen + C::kBarOffset);
   const uint32_t bar_full = smem_u32(&bars->full[0]);
   const uint32_t bar_empty = smem_u32(&bars->empty[0]);
   const uint32_t bar_tfull = smem_u32(&bars->tmem_full);
@@ -224,108 +329,185 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = CG == 1 ? 0u : cluster_ctarank();      // position inside the CTA pair
+  const bool leader = rank == 0;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar_full + 8 * s, 1);
+      // leader: its own producer's arrive + (CG == 2) the peer's "my half has landed" arrive
+      mbar_init(bar_full + 8 * s, leader ? CG : 1);
       mbar_init(bar_empty + 8 * s, 1);
     }
     mbar_init(bar_tfull, 1);
-    mbar_init(bar_tempty, kEpiWarps);
+    mbar_init(bar_tempty, kEpiWarps * CG);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tmap(&tm_a);
-    prefetch_tmap(&tm_b);
-    if (p.has_resid) prefetch_tmap(&tm_r);
+    prefetch_tmap(tm_a);
+    prefetch_tmap(tm_b);
+    if (p.has_resid) prefetch_tmap(tm_r);
   }
-  if (warp == 1) tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+  if (warp == 1) tmem_alloc<CG>(smem_u32(&bars->tmem_base), kTmemCols);
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();          // both CTAs' barriers exist before any remote arrive
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
-  const int m_tiles = p.header[kHdrMTiles];
-  const int total_tiles = m_tiles * p.n_tiles_n;
+  const int m_groups = p.header[kHdrMTiles] / CG;   // M-tiles come in groups of CG (same expert)
+  const int total_tiles = m_groups * p.n_tiles_n;
   const int kt_count = p.K >> 6;                    // scale atoms (K = 64 each) along K
-  const int k_stages = (kt_count + 3) >> 2;
+  const int k_stages = (kt_count + kKSteps - 1) / kKSteps;
   const bool resid = p.has_resid != 0;
+  const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ producer
-    if (lane == 0) {
+    // ------------------------------------------------------------ producer (whole warp, one lane issues)
+    {
+      const bool issuer = elect_one();
       uint32_t stage = 0, phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int mt = tile / p.n_tiles_n, nt = tile - mt * p.n_tiles_n;
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+        const int mg = tile / p.n_tiles_n, nt = tile - mg * p.n_tiles_n;
+        const int mt = mg * CG + (int)rank;
         const int e = p.tile_expert[mt];
         const int brow0 = e * p.b_rows_per_expert + nt * (EPI == kEpiSwiGLU ? 128 : 256);
         const int brow1 = brow0 + p.half1_row_offset;
         const bool half1 = (EPI == kEpiSwiGLU) || (nt * 256 + 128 < p.n_out);
         const int rt0 = (brow0 - e * p.b_rows_per_expert) >> 7, rt1 = (brow1 - e * p.b_rows_per_expert) >> 7;
         const uint8_t* bsf = p.b_sf + (size_t)e * p.b_sf_expert_stride;
+        const uint8_t* bsf0 = bsf + (size_t)rt0 * kt_count * 512u;
+        const uint8_t* bsf1 = bsf + (size_t)rt1 * kt_count * 512u;
+        const uint8_t* asf = p.a_sf + (size_t)mt * kt_count * 512u;
+        const uint8_t* rsf = p.r_sf + (size_t)mt * kt_count * 512u;
+        // weight rows this CTA keeps in shared memory
+        const bool load_b0 = CG == 1 || rank == 0;
+        const bool load_b1 = half1 && (CG == 1 || rank == 1);
+        const uint32_t data_bytes = kTileA + (resid ? kTileA : 0) + ((load_b0 ? 1 : 0) + (load_b1 ? 1 : 0)) * (kBM * kStageKBytes);
+        const uint32_t sf_count = 1u + (resid ? 1u : 0u) + (half1 ? 2u : 1u);
         for (int ks = 0; ks < k_stages; ++ks) {
           ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status);
           if (!ok) break;
-          const int atoms = min(4, kt_count - ks * 4);
+          const int atoms = min(kKSteps, kt_count - ks * kKSteps);
           const uint32_t sf_bytes = (uint32_t)atoms * 512u;
-          const uint32_t sbase = smem_base + stage * kStageBytes;
+          const uint32_t sbase = smem_base + stage * C::kStageBytes;
           const uint32_t full = bar_full + 8 * stage;
-          const uint32_t bytes = kTileA + (resid ? kTileA : 0) + (half1 ? kTileB : kTileB / 2) +
-                                 sf_bytes * (1u + (resid ? 1u : 0u) + (half1 ? 2u : 1u));
-          mbar_expect_tx(full, bytes);
-          tma_load_2d(sbase, &tm_a, ks * kStageKBytes, mt * kBM, full);
-          if (resid) tma_load_2d(sbase + kOffR, &tm_r, ks * kStageKBytes, mt * kBM, full);
-          tma_load_2d(sbase + kOffB, &tm_b, ks * kStageKBytes, brow0, full);
-          if (half1) tma_load_2d(sbase + kOffB + kTileB / 2, &tm_b, ks * kStageKBytes, brow1, full);
-          const size_t a_off = ((size_t)mt * kt_count + (size_t)ks * 4) * 512u;
-          bulk_load(sbase + kOffSfA, p.a_sf + a_off, sf_bytes, full);
-          if (resid) bulk_load(sbase + kOffSfR, p.r_sf + a_off, sf_bytes, full);
-          bulk_load(sbase + kOffSfB, bsf + ((size_t)rt0 * kt_count + (size_t)ks * 4) * 512u, sf_bytes, full);
-          if (half1)
-            bulk_load(sbase + kOffSfB + kSfA, bsf + ((size_t)rt1 * kt_count + (size_t)ks * 4) * 512u, sf_bytes, full);
+          const int kc = ks * kStageKBytes;
+          const size_t sf_off = (size_t)ks * (size_t)kSfA;
+          if (issuer) {
+            mbar_expect_tx(full, data_bytes + sf_bytes * sf_count);
+            tma_load_2d(sbase, tm_a, kc, mt * kBM, full);
+            if (resid) tma_load_2d(sbase + kOffR, tm_r, kc, mt * kBM, full);
+            if (load_b0) tma_load_2d(sbase + kOffB, tm_b, kc, brow0, full);
+            if (load_b1) tma_load_2d(sbase + kOffB + (CG == 1 ? kTileA : 0), tm_b, kc, brow1, full);
+            bulk_load(sbase + C::kOffSfA, asf + sf_off, sf_bytes, full);
+            if (resid) bulk_load(sbase + C::kOffSfR, rsf + sf_off, sf_bytes, full);
+            bulk_load(sbase + C::kOffSfB, bsf0 + sf_off, sf_bytes, full);
+            if (half1) bulk_load(sbase + C::kOffSfB + kSfA, bsf1 + sf_off, sf_bytes, full);
+            if ((p.dbg & 32) && ks + kStages < k_stages) {
+              // the same tile, kStages stages ahead: pull it into L2 now
+              const int kp = (ks + kStages) * kStageKBytes;
+              const size_t sp = (size_t)(ks + kStages) * (size_t)kSfA;
+              tma_prefetch_2d(tm_a, kp, mt * kBM);
+              if (resid) tma_prefetch_2d(tm_r, kp, mt * kBM);
+              if (load_b0) tma_prefetch_2d(tm_b, kp, brow0);
+              if (load_b1) tma_prefetch_2d(tm_b, kp, brow1);
+              bulk_prefetch(asf + sp, kSfA);
+              if (resid) bulk_prefetch(rsf + sp, kSfA);
+              bulk_prefetch(bsf0 + sp, kSfA);
+              if (half1) bulk_prefetch(bsf1 + sp, kSfA);
+            }
+          }
+          __syncwarp();
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
-      // drain: let every armed stage land before the CTA may exit
+      // drain: let every armed stage land and be consumed before the CTA may exit
       for (int s = 0; s < kStages && ok; ++s) {
         ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status);
         if (++stage == kStages) { stage = 0; phase ^= 1u; }
       }
     }
+  } else if (warp == 1 && !leader) {
+    // ------------------------------------------------------------ peer CTA: tell the leader when this
+    // CTA's half of a stage has landed (the leader issues the MMAs for both CTAs)
+    {
+      const bool issuer = elect_one();
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      const uint32_t leader_full = map_to_cta(bar_full, 0);
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+        for (int ks = 0; ks < k_stages; ++ks) {
+          ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status);
+          if (!ok) break;
+          if (issuer) mbar_arrive_remote(leader_full + 8 * stage);
+          __syncwarp();
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA; whole warp, one lane issues)
+    {
+      const bool issuer = elect_one();
       uint32_t stage = 0, phase = 0, kcount = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-        ok = mbar_wait(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status);
+      constexpr uint32_t idesc = idesc_nvf4<CG>();
+      // constant high words of the two descriptor kinds; the low word carries the address
+      // swizzled K-major operand tiles: 8-row groups 8 * row bytes apart; 128-byte rows use the
+      // 128-byte swizzle (type 2), 64-byte rows the 64-byte swizzle (type 4)
+      constexpr uint32_t kSw128Hi = (uint32_t)((8 * kStageKBytes) >> 4) | (1u << 14) | ((kStageKBytes == 128 ? 2u : 4u) << 29);
+      constexpr uint32_t kSfHi = (uint32_t)(128 >> 4) | (1u << 14);
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
+        ok = CG == 1 ? mbar_wait(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status)
+                     : mbar_wait_cluster(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
         for (int ks = 0; ks < k_stages; ++ks, ++kcount) {
-          ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status);
+          ok = CG == 1 ? mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status)
+                       : mbar_wait_cluster(bar_full + 8 * stage, phase, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          const int atoms = min(4, kt_count - ks * 4);
-          const uint32_t sbase = smem_base + stage * kStageBytes;
+          const int atoms = min(kKSteps, kt_count - ks * kKSteps);
+          const uint32_t sbase = smem_base + stage * C::kStageBytes;
           const uint32_t sfcol = tmem + kTmemSfBase + (kcount & 1u) * kTmemSfPerBuf;
-          for (int j = 0; j < atoms; ++j) {
-            tc_cp_sf(sfcol + 4 * j, desc_sf_atom(sbase + kOffSfA + 512 * j));
-            if (resid) tc_cp_sf(sfcol + 16 + 4 * j, desc_sf_atom(sbase + kOffSfR + 512 * j));
-            tc_cp_sf(sfcol + 32 + 8 * j, desc_sf_atom(sbase + kOffSfB + 512 * j));
-            tc_cp_sf(sfcol + 32 + 8 * j + 4, desc_sf_atom(sbase + kOffSfB + kSfA + 512 * j));
+          // descriptor low words: (address >> 4) [| LBO field for the swizzled operands]
+          const uint32_t a_lo = ((sbase & 0x3FFFFu) >> 4) | (1u << 16);
+          const uint32_t r_lo = (((sbase + kOffR) & 0x3FFFFu) >> 4) | (1u << 16);
+          const uint32_t b_lo = (((sbase + kOffB) & 0x3FFFFu) >> 4) | (1u << 16);
+          const uint32_t sfa_lo = ((sbase + C::kOffSfA) & 0x3FFFFu) >> 4;
+          const uint32_t sfr_lo = ((sbase + C::kOffSfR) & 0x3FFFFu) >> 4;
+          const uint32_t sfb_lo = ((sbase + C::kOffSfB) & 0x3FFFFu) >> 4;
+          const bool first = ks == 0;
+          if (issuer) {
+            if (!(p.dbg & 1)) {
+#pragma unroll
+              for (int j = 0; j < kKSteps; ++j) {
+                if (j < atoms) {
+                  tc_cp_sf<CG>(sfcol + 4 * j, ((uint64_t)kSfHi << 32) | (sfa_lo + 32 * j));
+                  if (resid) tc_cp_sf<CG>(sfcol + 4 * kKSteps + 4 * j, ((uint64_t)kSfHi << 32) | (sfr_lo + 32 * j));
+                  tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j, ((uint64_t)kSfHi << 32) | (sfb_lo + 32 * j));
+                  tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j + 4, ((uint64_t)kSfHi << 32) | (sfb_lo + (kSfA >> 4) + 32 * j));
+                }
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < kKSteps; ++j) {
+              if (j < ((p.dbg & 2) ? (first ? 1 : 0) : atoms)) {
+                const uint64_t bdesc = ((uint64_t)kSw128Hi << 32) | (b_lo + 2 * j);
+                tc_mma_nvf4<CG>(tmem, ((uint64_t)kSw128Hi << 32) | (a_lo + 2 * j), bdesc, idesc, sfcol + 4 * j,
+                                sfcol + 8 * kKSteps + 8 * j, (!first || j > 0) ? 1u : 0u);
+                if (resid)
+                  tc_mma_nvf4<CG>(tmem, ((uint64_t)kSw128Hi << 32) | (r_lo + 2 * j), bdesc, idesc,
+                                  sfcol + 4 * kKSteps + 4 * j, sfcol + 8 * kKSteps + 8 * j, 1u);
+              }
+            }
+            tc_commit<CG>(bar_empty + 8 * stage);
           }
-          for (int j = 0; j < atoms; ++j) {
-            const uint64_t bdesc = desc_sw128(sbase + kOffB + 32 * j);
-            tc_mma_nvf4(tmem, desc_sw128(sbase + 32 * j), bdesc, kIdesc, sfcol + 4 * j, sfcol + 32 + 8 * j,
-                        (ks > 0 || j > 0) ? 1u : 0u);
-            if (resid)
-              tc_mma_nvf4(tmem, desc_sw128(sbase + kOffR + 32 * j), bdesc, kIdesc, sfcol + 16 + 4 * j,
-                          sfcol + 32 + 8 * j, 1u);
-          }
-          tc_commit(bar_empty + 8 * stage);
+          __syncwarp();
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit(bar_tfull);
+        if (ok && issuer) tc_commit<CG>(bar_tfull);
+        __syncwarp();
       }
     }
   } else {
@@ -339,8 +521,10 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
                                      ? __fdiv_rn(__uint_as_float(p.a_amax_bits[0]), kGlobalDiv) : 1.0f);
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-      const int mt = tile / p.n_tiles_n, nt = tile - mt * p.n_tiles_n;
+    const uint32_t tempty_addr = CG == 1 ? bar_tempty : map_to_cta(bar_tempty, 0);
+    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
+      const int mg = tile / p.n_tiles_n, nt = tile - mg * p.n_tiles_n;
+      const int mt = mg * CG + (int)rank;
       const int e = p.tile_expert[mt];
       const bool valid = row_in_tile < p.tile_rows[mt];
       const int prow = mt * kBM + row_in_tile;
@@ -360,8 +544,12 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty);     // accumulator is free for the next tile
+      if (lane == 0) {                            // accumulator is free for the next tile
+        if (CG == 1) mbar_arrive(bar_tempty);
+        else mbar_arrive_remote(tempty_addr);
+      }
 
+      if (p.dbg & 4) continue;
       if (EPI == kEpiSwiGLU) {
         const float h_gs = p.h_gs[0];
         const int I = p.n_out;
@@ -452,22 +640,48 @@ gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const 
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();          // the peer may still be signalling this CTA's barriers
   tc_fence_after();
-  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 1) tmem_dealloc<CG>(tmem, kTmemCols);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_r,
+            const __grid_constant__ CUtensorMap tm_b) {
+  gemm_body<EPI, 1>(p, &tm_a, &tm_r, &tm_b);
+}
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_kernel_pair(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_r,
+                 const __grid_constant__ CUtensorMap tm_b) {
+  gemm_body<EPI, 2>(p, &tm_a, &tm_r, &tm_b);
 }
 
 }  // namespace
 
-quads_status launch_gemm(int epi, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
+quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
                          const CUtensorMap& tm_b, int n_sms, cudaStream_t stream) {
-  static bool attr_set[3] = {false, false, false};
-  void (*fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap) =
-      epi == kEpiStore ? gemm_kernel<kEpiStore> : (epi == kEpiSwiGLU ? gemm_kernel<kEpiSwiGLU> : gemm_kernel<kEpiCombine>);
-  if (!attr_set[epi]) {
-    QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    attr_set[epi] = true;
+  typedef void (*Fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap);
+  static bool attr_set[2][3] = {{false, false, false}, {false, false, false}};
+  Fn fn;
+  int smem;
+  if (cta_group == 2) {
+    fn = epi == kEpiStore ? gemm_kernel_pair<kEpiStore>
+                          : (epi == kEpiSwiGLU ? gemm_kernel_pair<kEpiSwiGLU> : gemm_kernel_pair<kEpiCombine>);
+    smem = Cfg<2>::kSmemBytes;
+  } else {
+    fn = epi == kEpiStore ? gemm_kernel<kEpiStore> : (epi == kEpiSwiGLU ? gemm_kernel<kEpiSwiGLU> : gemm_kernel<kEpiCombine>);
+    smem = Cfg<1>::kSmemBytes;
   }
-  fn<<<n_sms, kThreads, kSmemBytes, stream>>>(p, tm_a, tm_r, tm_b);
+  const int g = cta_group == 2 ? 1 : 0;
+  if (!attr_set[g][epi]) {
+    QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_set[g][epi] = true;
+  }
+  const int grid = cta_group == 2 ? (n_sms / 2) * 2 : n_sms;
+  fn<<<grid, kThreads, smem, stream>>>(p, tm_a, tm_r, tm_b);
   note_launch();
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;

@@ -9,6 +9,7 @@ namespace quads {
 constexpr int kRouteTokensPerCta = 32;
 constexpr int kMaxTopk = 16;
 constexpr int kMaxExperts = 256;
+constexpr int kMTileGroup = 2;   // every expert's padded rows are a multiple of 128 * kMTileGroup
 
 // header words written by the scan (device side sizes of the dispatch)
 enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, kHdrWords = 8 };
@@ -55,6 +56,11 @@ __global__ void dense_dispatch_kernel(int T, int32_t* pos_pad, int32_t* row_toke
                                       int32_t* tile_expert, int32_t* tile_rows, int32_t* header);
 
 // ---- gemm.cu
+#ifndef QUADS_GEMM_KSTEPS
+#define QUADS_GEMM_KSTEPS 4
+#endif
+constexpr int kGemmKSteps = QUADS_GEMM_KSTEPS;        // K = 64 MMAs per pipeline stage (2 or 4)
+constexpr int kGemmStageKBytes = 32 * kGemmKSteps;    // packed FP4 bytes per operand row per stage
 enum { kEpiStore = 0, kEpiSwiGLU = 1, kEpiCombine = 2 };
 
 struct GemmParams {
@@ -87,10 +93,11 @@ struct GemmParams {
   uint16_t* h_export;    // optional bf16 [A, n_out] in dispatch order
   const int32_t* tile_prefix;
   const int32_t* offsets;
+  int dbg;               // debugging bit mask (0 in normal operation)
   int32_t* status;       // device status word (QUADS_ERR_TIMEOUT on a failed wait)
 };
 
-quads_status launch_gemm(int epi, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
+quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
                          const CUtensorMap& tm_b, int n_sms, cudaStream_t stream);
 
 }  // namespace quads

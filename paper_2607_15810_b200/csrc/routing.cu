@@ -153,7 +153,7 @@ scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32
     for (int i = 0; i < E; ++i) {
       off[i] = a; tpre[i] = t;
       a += cnt[i];
-      t += (cnt[i] + 127) >> 7;
+      t += ((cnt[i] + 128 * kMTileGroup - 1) / (128 * kMTileGroup)) * kMTileGroup;
     }
     off[E] = a; tpre[E] = t;
     header[kHdrMTiles] = t;
@@ -170,7 +170,7 @@ scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32
     const int n_t = tpre[e + 1] - tpre[e];
     for (int m = lane; m < n_t; m += 32) {
       tile_expert[tpre[e] + m] = e;
-      tile_rows[tpre[e] + m] = min(128, cnt[e] - m * 128);
+      tile_rows[tpre[e] + m] = max(0, min(128, cnt[e] - m * 128));
     }
   }
 }
@@ -222,9 +222,9 @@ dense_dispatch_kernel(int T, int32_t* __restrict__ pos_pad, int32_t* __restrict_
                       float* __restrict__ row_weight, int32_t* __restrict__ tile_expert,
                       int32_t* __restrict__ tile_rows, int32_t* __restrict__ header) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  const int m_tiles = (T + 127) >> 7;
+  const int m_tiles = ((T + 128 * kMTileGroup - 1) / (128 * kMTileGroup)) * kMTileGroup;
   if (i < T) { pos_pad[i] = i; row_token[i] = i; row_weight[i] = 1.f; }
-  if (i < m_tiles) { tile_expert[i] = 0; tile_rows[i] = min(128, T - i * 128); }
+  if (i < m_tiles) { tile_expert[i] = 0; tile_rows[i] = max(0, min(128, T - i * 128)); }
   if (i == 0) { header[kHdrMTiles] = m_tiles; header[kHdrPaddedRows] = m_tiles * 128; header[kHdrAssignments] = T; }
 }
 

@@ -110,10 +110,10 @@ size_t quads_fake_quant_workspace_bytes(int64_t n_tensors);
  * trainer whose device memory belongs entirely to its own caching pool, a
  * plugin that is forbidden to allocate after start-up, or code on a path where
  * the implicit device synchronisation of an allocation is not acceptable.  For
- * them this entry point takes no workspace: its scratch, one 4-byte amax word
- * per tensor, is a fixed array of QUADS_NOALLOC_MAX_TENSORS words inside the
- * library image (16 KiB, resident on every GPU that loads the library until the
- * process exits).  Arguments, outputs and results are those of
+ * them this entry point takes no workspace: its scratch, two 4-byte words per
+ * tensor (the running amax and an arrival counter), is a fixed array sized for
+ * QUADS_NOALLOC_MAX_TENSORS tensors inside the library image (32 KiB, resident
+ * on every GPU that loads the library until the process exits).  Arguments, outputs and results are those of
  * quads_fake_quant_weights, bit for bit.
  *   - n_tensors > QUADS_NOALLOC_MAX_TENSORS returns QUADS_ERR_LIMIT and
  *     launches nothing; split the batch.

@@ -224,7 +224,7 @@ size_t quads_sf_tiled_bytes(int64_t rows, int64_t K) {
 
 size_t quads_quantize_workspace_bytes(void) { return 256; }
 size_t quads_fake_quant_workspace_bytes(int64_t n_tensors) {
-  return align_up((size_t)(n_tensors > 0 ? n_tensors : 1) * 4, 256);
+  return align_up((size_t)(n_tensors > 0 ? n_tensors : 1) * 8, 256);
 }
 int32_t quads_last_launch_count(void) { return g_launch_count; }
 
@@ -244,26 +244,33 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   quads_status s = device_info(&di);
   if (s != QUADS_OK) return s;
   if (n_tensors == 0) return QUADS_OK;
+  // scratch: one amax word and one arrival counter per tensor, zero on entry
   uint32_t* amax_bits = static_cast<uint32_t*>(workspace);
-  if (!gs_in) {
-    QUADS_CUDA_OK(cudaMemsetAsync(amax_bits, 0, (size_t)n_tensors * 4, st));
-    if (rows > 0) {
-      const int64_t chunks = rows * (K / 8);
-      int gx = (int)((chunks + 256 * 8 - 1) / (256 * 8));
-      const int cap = (di.sm_count * 8 + (int)n_tensors - 1) / (int)n_tensors;
-      if (gx > cap) gx = cap;
-      if (gx < 1) gx = 1;
-      amax_kernel<<<dim3(gx, (unsigned)n_tensors), 256, 0, st>>>(static_cast<const uint16_t*>(x), rows, K, ld,
-                                                                   tensor_stride, amax_bits);
-      note_launch();
-    }
-  }
+  uint32_t* counters = amax_bits + n_tensors;
+  if (!gs_in) QUADS_CUDA_OK(cudaMemsetAsync(amax_bits, 0, (size_t)n_tensors * 8, st));
+  const uint16_t* xp = static_cast<const uint16_t*>(x);
+  uint16_t* fqp = static_cast<uint16_t*>(fq);
+  int nt = (int)n_tensors;
+  int tiled = sf_layout == QUADS_SF_TILED;
+  int64_t sf_stride = tiled ? (int64_t)quads_sf_tiled_bytes(rows, K) : rows * (K / 16);
   const int64_t nblk = rows * (K / 16);
-  const unsigned gx = (unsigned)((nblk + 255) / 256);
-  const int64_t sf_stride = sf_layout == QUADS_SF_TILED ? (int64_t)quads_sf_tiled_bytes(rows, K) : rows * (K / 16);
-  quantize_kernel<<<dim3(gx > 0 ? gx : 1, (unsigned)n_tensors), 256, 0, st>>>(
-      static_cast<const uint16_t*>(x), rows, K, ld, tensor_stride, gs_in, amax_bits, q, sf,
-      static_cast<uint16_t*>(fq), gs_out, sf_layout == QUADS_SF_TILED, sf_stride);
+  static int blocks_per_sm = 0;
+  if (blocks_per_sm == 0) {
+    int b = 0;
+    QUADS_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, fused_quantize_kernel, 256, 0));
+    blocks_per_sm = b < 1 ? 1 : (b > 8 ? 8 : b);
+  }
+  int max_groups = 4;
+  { const char* e = getenv("QUADS_FQ_GROUPS"); if (e) max_groups = atoi(e); }
+  int n_groups = n_tensors < max_groups ? (int)n_tensors : max_groups;
+  int64_t want = (nblk * n_groups + 255) / 256;            // no more CTAs than there is work
+  int grid = di.sm_count * blocks_per_sm;
+  if (want < grid) grid = (int)want;
+  if (grid < n_groups) grid = n_groups;
+  void* args[] = {&xp, &rows, &K, &ld, &tensor_stride, &nt, &gs_in, &amax_bits, &counters, &q, &sf, &fqp,
+                  &gs_out, &tiled, &sf_stride, &n_groups};
+  QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fused_quantize_kernel), dim3(grid), dim3(256),
+                                            args, 0, st));
   note_launch();
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
@@ -286,7 +293,7 @@ quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t 
 }
 
 // ---------------------------------------------------------------------------
-// Allocation-free fake-quant.  Its scratch (one amax word per tensor) lives in
+// Allocation-free fake-quant.  Its scratch (an amax word and an arrival counter per tensor) lives in
 // the library image, so a caller that must not allocate device memory -- for
 // instance code running under a memory pool it does not own, or inside a
 // region where cudaMalloc's implicit device synchronisation is forbidden --
@@ -294,7 +301,7 @@ quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t 
 // symbol; the device address comes from cudaGetSymbolAddress, looked up once
 // per device with that device current.
 // ---------------------------------------------------------------------------
-static __device__ __align__(256) uint32_t g_noalloc_amax[QUADS_NOALLOC_MAX_TENSORS];
+static __device__ __align__(256) uint32_t g_noalloc_amax[2 * QUADS_NOALLOC_MAX_TENSORS];
 
 static quads_status noalloc_scratch(uint32_t** out) {
   static std::mutex mu;
@@ -320,10 +327,10 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
   uint32_t* scratch = nullptr;
   quads_status s = noalloc_scratch(&scratch);
   if (s != QUADS_OK) return s;
-  // quantize_common zeroes the amax words it is about to use on the stream
-  // before the reduction, so the previous call's contents never leak in.
+  // quantize_common zeroes the words it is about to use on the stream before
+  // the kernel, so the previous call's contents never leak in.
   return quantize_common(w, n_tensors, N, K, K, N * K, nullptr, w_fq, q, sf, gs, sf_layout, scratch,
-                         sizeof(uint32_t) * QUADS_NOALLOC_MAX_TENSORS, static_cast<cudaStream_t>(cuda_stream));
+                         sizeof(uint32_t) * 2 * QUADS_NOALLOC_MAX_TENSORS, static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t quads_moe_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk, int32_t N) {

@@ -17,9 +17,10 @@ enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, 
 // ---- quantize.cu
 __global__ void amax_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
                             uint32_t* amax_bits);
-__global__ void quantize_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
-                                const float* gs_in, const uint32_t* amax_bits, uint8_t* q, uint8_t* sf,
-                                uint16_t* fq, float* gs_out, int sf_tiled, int64_t sf_tensor_stride);
+__global__ void fused_quantize_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
+                                      int n_tensors, const float* gs_in, uint32_t* amax_bits, uint32_t* counters,
+                                      uint8_t* q, uint8_t* sf, uint16_t* fq, float* gs_out, int sf_tiled,
+                                      int64_t sf_tensor_stride, int n_groups);
 __global__ void rac_stats_kernel(const uint16_t* x, int T, int H, const float* gs_in, const uint32_t* amax_bits,
                                  float* gs_store, int rows_per_cta, float* partials, uint8_t* xq_out,
                                  uint8_t* xsf_out);

@@ -65,48 +65,155 @@ __device__ __forceinline__ float gs_from_amax_bits(uint32_t bits) {
 }
 
 // ---------------------------------------------------------------------------
-// NVFP4 quantize / fake-quant: one thread per 16-element block.
-// gridDim.y = tensor.  The per-tensor scale comes from gs_in[tensor] when
-// gs_in != NULL, else from amax_bits[tensor].
+// Fused amax + NVFP4 quantize / fake-quant in ONE cooperative launch.
+// The CTAs form `n_groups` groups (CTA c belongs to group c % n_groups, so every
+// group spans all SMs).  A group takes tensors group, group + n_groups, ...:
+//   phase 1  its CTAs stream the tensor once (kept in L2: evict_last), reduce
+//            |x| max, publish it with atomicMax and meet at a per-tensor counter;
+//   phase 2  they read the tensor again (from L2), quantize, and stream the
+//            outputs out (evict_first).
+// Other groups overlap their phases with this group's barrier wait.  DRAM sees
+// each input byte once: 2 B read + the outputs per element.
+// `amax_bits` and `counters` (one word each per tensor) must be zero on entry.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
-                const float* __restrict__ gs_in, const uint32_t* __restrict__ amax_bits,
-                uint8_t* __restrict__ q, uint8_t* __restrict__ sf, uint16_t* __restrict__ fq,
-                float* __restrict__ gs_out, int sf_tiled, int64_t sf_tensor_stride) {
-  const int t = blockIdx.y;
-  const float gs = gs_in ? gs_in[t] : gs_from_amax_bits(amax_bits[t]);
-  if (gs_out && blockIdx.x == 0 && threadIdx.x == 0) gs_out[t] = gs;
+__device__ __forceinline__ void ldg256_keep(const void* p, uint4& a, uint4& b) {
+  asm volatile("ld.global.L2::evict_last.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p));
+}
+__device__ __forceinline__ void ldg256_stream(const void* p, uint4& a, uint4& b) {
+  asm volatile("ld.global.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p));
+}
+__device__ __forceinline__ uint32_t absmax8(const uint4& v) {
+  return __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
+}
+
+__global__ void __launch_bounds__(256, 4)
+fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
+                      int n_tensors, const float* __restrict__ gs_in, uint32_t* __restrict__ amax_bits,
+                      uint32_t* __restrict__ counters, uint8_t* __restrict__ q, uint8_t* __restrict__ sf,
+                      uint16_t* __restrict__ fq, float* __restrict__ gs_out, int sf_tiled, int64_t sf_tensor_stride,
+                      int n_groups) {
+  const int group = blockIdx.x % n_groups;
+  const int rank = blockIdx.x / n_groups;
+  const int gsize = ((int)gridDim.x - group + n_groups - 1) / n_groups;
   const int64_t k16 = K >> 4;
   const int64_t nblk = rows * k16;
-  const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= nblk) return;
-  const int64_t r = b / k16, kb = b - r * k16;
-  const uint16_t* src = x + (size_t)t * tensor_stride + r * ld + kb * 16;
-  uint4 v0, v1;
-  ldg256(src, v0, v1);
-  float f[16];
-  unpack8(v0, f);
-  unpack8(v1, f + 8);
-  const BlockQ bq = quantize_block(f, gs);
-  const size_t row_global = (size_t)t * rows + r;
-  if (q) *reinterpret_cast<uint2*>(q + row_global * (K >> 1) + kb * 8) = make_uint2(bq.lo, bq.hi);
-  if (sf) {
-    uint8_t* sft = sf + (size_t)t * sf_tensor_stride;
-    if (sf_tiled) sft[sf_tiled_offset(r, kb, (K + 63) >> 6)] = (uint8_t)bq.sf8;
-    else sft[r * k16 + kb] = (uint8_t)bq.sf8;
-  }
-  if (fq) {
-    float o[16];
-    dequant_block(bq, o);
-    uint4 w0, w1;
-    w0.x = f32x2_to_bf16x2(o[0], o[1]);   w0.y = f32x2_to_bf16x2(o[2], o[3]);
-    w0.z = f32x2_to_bf16x2(o[4], o[5]);   w0.w = f32x2_to_bf16x2(o[6], o[7]);
-    w1.x = f32x2_to_bf16x2(o[8], o[9]);   w1.y = f32x2_to_bf16x2(o[10], o[11]);
-    w1.z = f32x2_to_bf16x2(o[12], o[13]); w1.w = f32x2_to_bf16x2(o[14], o[15]);
-    uint4* dst = reinterpret_cast<uint4*>(fq + (size_t)t * rows * K + r * K + kb * 16);
-    dst[0] = w0;
-    dst[1] = w1;
+  const int64_t gthreads = (int64_t)gsize * blockDim.x;
+  const int64_t gtid = (int64_t)rank * blockDim.x + threadIdx.x;
+  __shared__ uint32_t wmax[8];
+  __shared__ float gs_sh;
+  for (int t = group; t < n_tensors; t += n_groups) {
+    const uint16_t* base = x + (size_t)t * tensor_stride;
+    float gs;
+    if (gs_in) {
+      gs = gs_in[t];
+    } else {
+      // ---- phase 1: tensor amax, one 32-byte block per load
+      uint32_t m = 0;
+      if (ld == K) {
+        int64_t b = gtid;
+        for (; b + 3 * gthreads < nblk; b += 4 * gthreads) {
+          uint4 a0, a1, b0, b1, c0, c1, d0, d1;
+          ldg256_keep(base + b * 16, a0, a1);
+          ldg256_keep(base + (b + gthreads) * 16, b0, b1);
+          ldg256_keep(base + (b + 2 * gthreads) * 16, c0, c1);
+          ldg256_keep(base + (b + 3 * gthreads) * 16, d0, d1);
+          m = __vmaxu2(m, __vmaxu2(__vmaxu2(__vmaxu2(absmax8(a0), absmax8(a1)), __vmaxu2(absmax8(b0), absmax8(b1))),
+                                   __vmaxu2(__vmaxu2(absmax8(c0), absmax8(c1)), __vmaxu2(absmax8(d0), absmax8(d1)))));
+        }
+        for (; b < nblk; b += gthreads) {
+          uint4 a0, a1;
+          ldg256_keep(base + b * 16, a0, a1);
+          m = __vmaxu2(m, __vmaxu2(absmax8(a0), absmax8(a1)));
+        }
+      } else {
+        for (int64_t b = gtid; b < nblk; b += gthreads) {
+          const int64_t r = b / k16, kb = b - r * k16;
+          uint4 a0, a1;
+          ldg256_keep(base + r * ld + kb * 16, a0, a1);
+          m = __vmaxu2(m, __vmaxu2(absmax8(a0), absmax8(a1)));
+        }
+      }
+      uint32_t sm = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sm = max(sm, __shfl_xor_sync(0xFFFFFFFFu, sm, o));
+      if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = sm;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        uint32_t tm = 0;
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tm = max(tm, wmax[i]);
+        if (tm) atomicMax(amax_bits + t, tm << 16);
+        __threadfence();
+        atomicAdd(counters + t, 1u);
+        // bounded wait for the rest of the group (cooperative launch: all CTAs are resident)
+        const long long t0 = clock64();
+        while (atomicAdd(counters + t, 0u) < (uint32_t)gsize) {
+          __nanosleep(64);
+          if (clock64() - t0 > 4000000000ll) break;
+        }
+        __threadfence();
+        gs_sh = gs_from_amax_bits(atomicAdd(amax_bits + t, 0u));
+      }
+      __syncthreads();
+      gs = gs_sh;
+      __syncthreads();
+    }
+    if (gs_out && rank == 0 && threadIdx.x == 0) gs_out[t] = gs;
+    // ---- phase 2: quantize (16-element blocks), stream the outputs
+    uint8_t* qt = q ? q + (size_t)t * rows * (K >> 1) : nullptr;
+    uint8_t* sft = sf ? sf + (size_t)t * sf_tensor_stride : nullptr;
+    uint16_t* fqt = fq ? fq + (size_t)t * rows * K : nullptr;
+    const int kt_count = (int)((K + 63) >> 6);
+    const bool contiguous = (ld == K);
+    const uint32_t k16u = (uint32_t)k16;
+    auto emit = [&](int64_t b, const uint4& v0, const uint4& v1) {
+      float f[16];
+      unpack8(v0, f);
+      unpack8(v1, f + 8);
+      const BlockQ bq = quantize_block(f, gs);
+      // outputs are contiguous per tensor: block b owns bytes [8b, 8b+8) of q and [32b, 32b+32) of fq
+      if (qt) __stcs(reinterpret_cast<uint2*>(qt + b * 8), make_uint2(bq.lo, bq.hi));
+      if (sft) {
+        if (sf_tiled) {
+          const uint32_t r = (uint32_t)(b / k16u), kb = (uint32_t)(b - (int64_t)r * k16u);
+          sft[sf_tiled_offset(r, kb, kt_count)] = (uint8_t)bq.sf8;
+        } else {
+          sft[b] = (uint8_t)bq.sf8;
+        }
+      }
+      if (fqt) {
+        float o[16];
+        dequant_block(bq, o);
+        uint4* dst = reinterpret_cast<uint4*>(fqt + b * 16);
+        __stcs(dst, make_uint4(f32x2_to_bf16x2(o[0], o[1]), f32x2_to_bf16x2(o[2], o[3]),
+                               f32x2_to_bf16x2(o[4], o[5]), f32x2_to_bf16x2(o[6], o[7])));
+        __stcs(dst + 1, make_uint4(f32x2_to_bf16x2(o[8], o[9]), f32x2_to_bf16x2(o[10], o[11]),
+                                   f32x2_to_bf16x2(o[12], o[13]), f32x2_to_bf16x2(o[14], o[15])));
+      }
+    };
+    auto src_of = [&](int64_t b) -> const uint16_t* {
+      if (contiguous) return base + b * 16;
+      const int64_t r = b / k16, kb = b - r * k16;
+      return base + r * ld + kb * 16;
+    };
+    int64_t b = gtid;
+    for (; b + 3 * gthreads < nblk; b += 4 * gthreads) {     // four loads in flight per thread
+      uint4 a0, a1, c0, c1, d0, d1, e0, e1;
+      ldg256_stream(src_of(b), a0, a1);
+      ldg256_stream(src_of(b + gthreads), c0, c1);
+      ldg256_stream(src_of(b + 2 * gthreads), d0, d1);
+      ldg256_stream(src_of(b + 3 * gthreads), e0, e1);
+      emit(b, a0, a1);
+      emit(b + gthreads, c0, c1);
+      emit(b + 2 * gthreads, d0, d1);
+      emit(b + 3 * gthreads, e0, e1);
+    }
+    for (; b < nblk; b += gthreads) {
+      uint4 a0, a1;
+      ldg256_stream(src_of(b), a0, a1);
+      emit(b, a0, a1);
+    }
   }
 }
 

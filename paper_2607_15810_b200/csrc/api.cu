@@ -76,7 +76,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 struct MoeLayout {
   size_t header, amax, counters13, counters2, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
   size_t perm, pos_pad, row_token, row_weight;
-  size_t partials13, scores13, keys13, keys2, sel13, mask13, xq_pad, xsf, rq_pad, rsf;
+  size_t partials13, scores13, keys13, keys2, sel13, mask13, xq_tok, xsf_tok, rq_tok, rsf_tok, xq_pad, xsf, rq_pad, rsf;
   size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad;
   size_t total;
   int n_chunks, m_tiles_max, stats_ctas, rows_per_cta;
@@ -119,6 +119,10 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   L.keys13 = take((size_t)H * 8);
   L.sel13 = take((size_t)H * 4);
   L.mask13 = take((size_t)H);
+  L.xq_tok = take((size_t)T * (H / 2));
+  L.xsf_tok = take((size_t)T * (H / 16));
+  L.rq_tok = take((size_t)T * (H / 2));
+  L.rsf_tok = take((size_t)T * (H / 16));
   L.xq_pad = take(pad_rows * (H / 2));
   L.xsf = take((size_t)L.m_tiles_max * (H / 64) * 512);
   L.rq_pad = take(pad_rows * (H / 2));
@@ -163,6 +167,30 @@ inline void trace_mark(const char* name, cudaStream_t st) {
   g_trace.name[g_trace.n] = name;
   cudaEventRecord(g_trace.ev[g_trace.n], st);
   ++g_trace.n;
+}
+
+// Side stream on which the routing chain (route -> scan -> permute) runs next to the
+// activation chain (amax -> quantize -> select); both are joined before the dispatch copy.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool ok = false;
+};
+std::mutex g_side_mu;
+SideStream* side_stream() {
+  static SideStream per_device[64];
+  static const bool disabled = [] { const char* e = getenv("QUADS_NO_OVERLAP"); return e && e[0] == '1'; }();
+  if (disabled) return nullptr;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  SideStream& s = per_device[dev];
+  if (!s.ok) {
+    if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    s.ok = true;
+  }
+  return &s;
 }
 
 // 1: single-CTA tiles of 128 x 256 (default, the faster one as measured); 2: CTA pairs computing
@@ -437,6 +465,38 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, L.ids, st));
   trace_mark("memset", st);
 
+  // ---- routing and dispatch order: on a side stream, next to the activation chain below
+  std::unique_lock<std::mutex> side_lock(g_side_mu, std::defer_lock);
+  SideStream* side = (dense || g_trace.enabled) ? nullptr : side_stream();
+  cudaStream_t rs = st;
+  if (side) {
+    side_lock.lock();                       // event record / wait pairs of two host threads must not interleave
+    QUADS_CUDA_OK(cudaEventRecord(side->fork, st));
+    QUADS_CUDA_OK(cudaStreamWaitEvent(side->stream, side->fork, 0));
+    rs = side->stream;
+  }
+  if (dense) {
+    dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, pos_pad, row_token, row_weight, tile_expert,
+                                                           tile_rows, header);
+    note_launch();
+  } else {
+    int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
+    int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
+    route_kernel<<<L.n_chunks, 256, 0, rs>>>(a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts,
+                                              a->topk_ids, a->topk_w);
+    note_launch();
+    trace_mark("route", st);
+    scan_kernel<<<1, 1024, 0, rs>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
+                                   tile_rows, header, a->expert_offsets);
+    note_launch();
+    trace_mark("scan", st);
+    permute_kernel<<<(L.n_chunks + 3) / 4, 128, 0, rs>>>(T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets,
+                                                         tile_prefix, perm, pos_pad, row_token, row_weight, a->perm);
+    note_launch();
+  }
+  if (side) QUADS_CUDA_OK(cudaEventRecord(side->join, side->stream));
+  trace_mark("permute", st);
+
   // ---- per-tensor scale of x
   if (!a->a13_gs) {
     const int64_t chunks = (int64_t)T * (H / 8);
@@ -445,40 +505,14 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     amax_kernel<<<dim3(gx, 1), 256, 0, st>>>(x, T, H, H, 0, amax_bits);
     note_launch();
   }
-
   trace_mark("amax", st);
-  // ---- routing and dispatch order
-  if (dense) {
-    dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, pos_pad, row_token, row_weight, tile_expert,
-                                                           tile_rows, header);
-    note_launch();
-  } else {
-    int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
-    int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
-    route_kernel<<<L.n_chunks, 256, 0, st>>>(a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts,
-                                              a->topk_ids, a->topk_w);
-    note_launch();
-    trace_mark("route", st);
-    scan_kernel<<<1, 1024, 0, st>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
-                                   tile_rows, header, a->expert_offsets);
-    note_launch();
-    trace_mark("scan", st);
-    permute_kernel<<<(L.n_chunks + 3) / 4, 128, 0, st>>>(T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm,
-                                               pos_pad, row_token, row_weight, a->perm);
-    note_launch();
-  }
-
-  trace_mark("permute", st);
-  // ---- site 13: statistics, selection, quantize + residual + dispatch scatter
+  // ---- site 13: quantize (+ residual + statistics), selection, dispatch scatter
   const int nsel13 = a->rac_nsel_13;
-  float* gs13_store = a->a13_gs_out;
   uint8_t* mask13 = P(L.mask13);
-  if (nsel13 > 0 || a->xq || a->xsf || gs13_store) {
-    rac_stats_kernel<<<L.stats_ctas, H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32, 0, st>>>(
-        x, T, H, a->a13_gs, amax_bits, gs13_store, L.rows_per_cta, reinterpret_cast<float*>(P(L.partials13)),
-        a->xq, a->xsf);
-    note_launch();
-  }
+  rac_quant_kernel<<<L.stats_ctas, H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32, 0, st>>>(
+      x, T, H, a->a13_gs, amax_bits, a->a13_gs_out, L.rows_per_cta, nsel13 > 0 ? 1 : 0,
+      reinterpret_cast<float*>(P(L.partials13)), P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), a->xq, a->xsf);
+  note_launch();
   trace_mark("rac_stats", st);
   if (nsel13 > 0) {
     s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
@@ -487,14 +521,17 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     if (s != QUADS_OK) return s;
   }
   trace_mark("select13", st);
+  if (side) {
+    QUADS_CUDA_OK(cudaStreamWaitEvent(st, side->join, 0));
+    side_lock.unlock();
+  }
   {
-    const int64_t groups = (int64_t)T * (H / 64);
-    rac_dispatch_kernel<<<(unsigned)((groups + 255) / 256), 256, 0, st>>>(
-        x, T, H, a->a13_gs, amax_bits, nsel13, mask13, topk, pos_pad, P(L.xq_pad), P(L.xsf), P(L.rq_pad),
-        P(L.rsf), a->rq, a->rsf);
+    const int64_t chunks = (int64_t)T * (H / 32);
+    rac_scatter_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(
+        T, H, nsel13 > 0 ? 1 : 0, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok),
+        P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf);
     note_launch();
   }
-
   trace_mark("rac_dispatch", st);
   // ---- tensor maps
   CUtensorMap tm_x, tm_r, tm_w13;

@@ -21,20 +21,19 @@ __global__ void fused_quantize_kernel(const uint16_t* x, int64_t rows, int64_t K
                                       int n_tensors, const float* gs_in, uint32_t* amax_bits, uint32_t* counters,
                                       uint8_t* q, uint8_t* sf, uint16_t* fq, float* gs_out, int sf_tiled,
                                       int64_t sf_tensor_stride, int n_groups);
-__global__ void rac_stats_kernel(const uint16_t* x, int T, int H, const float* gs_in, const uint32_t* amax_bits,
-                                 float* gs_store, int rows_per_cta, float* partials, uint8_t* xq_out,
-                                 uint8_t* xsf_out);
+__global__ void rac_quant_kernel(const uint16_t* x, int T, int H, const float* gs_in, const uint32_t* amax_bits,
+                                 float* gs_store, int rows_per_cta, int with_residual, float* partials, uint8_t* xq,
+                                 uint8_t* xsf, uint8_t* rq, uint8_t* rsf, uint8_t* xq_exp, uint8_t* xsf_exp);
 constexpr int kScoreSlices = 16;
 __global__ void score_reduce_kernel(const float* partials, const int* n_part_ptr, int n_part_mul,
                                     int n_part_fixed, int C, double* slice_sums, unsigned int* counters,
                                     unsigned long long* score_keys);
 __global__ void rank_select_kernel(const unsigned long long* score_keys, int C, int n_sel, uint8_t* mask);
 __global__ void sel_list_kernel(const uint8_t* mask, int C, int32_t* sel_export);
-__global__ void rac_dispatch_kernel(const uint16_t* x, int T, int H, const float* gs_in,
-                                    const uint32_t* amax_bits, int n_sel,
-                                    const uint8_t* mask, int topk, const int32_t* pos_pad, uint8_t* xq_pad,
-                                    uint8_t* xsf_tiled, uint8_t* rq_pad, uint8_t* rsf_tiled, uint8_t* rq_out,
-                                    uint8_t* rsf_out);
+__global__ void rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* mask, int topk,
+                                   const int32_t* pos_pad, const uint8_t* xq, const uint8_t* xsf, const uint8_t* rq,
+                                   const uint8_t* rsf, uint8_t* xq_pad, uint8_t* xsf_tiled, uint8_t* rq_pad,
+                                   uint8_t* rsf_tiled, uint8_t* rq_exp, uint8_t* rsf_exp);
 __global__ void mask_codes_kernel(uint8_t* codes, const int* n_rows_ptr, int C, const uint8_t* mask);
 __global__ void combine_kernel(const uint16_t* y_pad, const int32_t* pos_pad, const float* wts, int T, int H,
                                int topk, uint16_t* out);

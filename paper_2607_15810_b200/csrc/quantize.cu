@@ -218,16 +218,20 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
 }
 
 // ---------------------------------------------------------------------------
-// RAC statistics at an activation site (Eq. channel-score): per-channel sum of
-// squared residuals of Q_A(x) over the rows this CTA owns, written as one
-// partial row per CTA (reduced later in a fixed order).  Optionally exports the
-// codes / scales of Q_A(x) in token order.
+// Site-13 quantization pass, token order.  For every row and 16-channel block:
+// Q_A(x) codes + scale; the residual Q_A(x) - x in float32 (Eq. residual-def);
+// its squared sum per channel over the rows this CTA owns (Eq. channel-score,
+// one partial row per CTA, reduced later in a fixed order); and the residual's
+// own quantization with the same per-tensor scale (the mask of Eq.
+// residual-recon is applied later, when rows are copied into dispatch order:
+// quantizing the residual does not depend on the selection).
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-rac_stats_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __restrict__ gs_in,
-                 const uint32_t* __restrict__ amax_bits, float* __restrict__ gs_store,
-                 int rows_per_cta, float* __restrict__ partials, uint8_t* __restrict__ xq_out,
-                 uint8_t* __restrict__ xsf_out) {
+rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __restrict__ gs_in,
+                 const uint32_t* __restrict__ amax_bits, float* __restrict__ gs_store, int rows_per_cta,
+                 int with_residual, float* __restrict__ partials, uint8_t* __restrict__ xq,
+                 uint8_t* __restrict__ xsf, uint8_t* __restrict__ rq, uint8_t* __restrict__ rsf,
+                 uint8_t* __restrict__ xq_exp, uint8_t* __restrict__ xsf_exp) {
   const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
   if (gs_store && blockIdx.x == 0 && threadIdx.x == 0) gs_store[0] = gs;
   const int k16 = H >> 4;
@@ -244,20 +248,30 @@ rac_stats_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
       unpack8(v0, f);
       unpack8(v1, f + 8);
       const BlockQ bq = quantize_block(f, gs);
-      dequant_block(bq, o);
+      const size_t qo = (size_t)r * (H >> 1) + kb * 8, so = (size_t)r * k16 + kb;
+      *reinterpret_cast<uint2*>(xq + qo) = make_uint2(bq.lo, bq.hi);
+      xsf[so] = (uint8_t)bq.sf8;
+      if (xq_exp) *reinterpret_cast<uint2*>(xq_exp + qo) = make_uint2(bq.lo, bq.hi);
+      if (xsf_exp) xsf_exp[so] = (uint8_t)bq.sf8;
+      if (with_residual) {
+        dequant_block(bq, o);
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const float d = __fsub_rn(o[i], f[i]);
-        acc[i] = __fmaf_rn(d, d, acc[i]);
+        for (int i = 0; i < 16; ++i) {
+          o[i] = __fsub_rn(o[i], f[i]);
+          acc[i] = __fmaf_rn(o[i], o[i], acc[i]);
+        }
+        const BlockQ br = quantize_block(o, gs);
+        *reinterpret_cast<uint2*>(rq + qo) = make_uint2(br.lo, br.hi);
+        rsf[so] = (uint8_t)br.sf8;
       }
-      if (xq_out) *reinterpret_cast<uint2*>(xq_out + (size_t)r * (H >> 1) + kb * 8) = make_uint2(bq.lo, bq.hi);
-      if (xsf_out) xsf_out[(size_t)r * k16 + kb] = (uint8_t)bq.sf8;
     }
-    float4* dst = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * H + kb * 16);
-    dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-    dst[2] = make_float4(acc[8], acc[9], acc[10], acc[11]);
-    dst[3] = make_float4(acc[12], acc[13], acc[14], acc[15]);
+    if (with_residual) {
+      float4* dst = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * H + kb * 16);
+      dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+      dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+      dst[2] = make_float4(acc[8], acc[9], acc[10], acc[11]);
+      dst[3] = make_float4(acc[12], acc[13], acc[14], acc[15]);
+    }
   }
 }
 
@@ -352,12 +366,12 @@ sel_list_kernel(const uint8_t* __restrict__ mask, int C, int32_t* __restrict__ s
 }
 
 // ---------------------------------------------------------------------------
-// Site-13 dispatch: for token row t and a group of four scale blocks (64
-// channels) recompute Q_A(x), form the residual, quantize it with the same
-// per-tensor scale, clear unselected channels (Eq. residual-recon), and write
-// both into every dispatched copy of the row (padded dispatch order, tiled
-// scale layout).  Residual codes are stored NEGATED (sign bit flipped) so the
-// GEMM can accumulate W Q(x) + W (-M Q(dx)) with two plain MMAs.
+// Site-13 dispatch: copy every token row's codes and scales into each of its
+// dispatched copies (padded dispatch order, tiled scale layout).  The residual
+// is masked on the way (Eq. residual-recon: codes of unselected channels are
+// cleared) and stored NEGATED (sign bits flipped) so that the GEMM can
+// accumulate W Q(x) + W (-M Q(dx)) with two plain MMAs.  Pure data movement:
+// one thread per (token, 32 channels = 16 code bytes).
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t nibble_mask8(const uint8_t* m) {
   // m[0..7] in {0,1} -> 0xF per selected nibble
@@ -372,57 +386,47 @@ __device__ __forceinline__ uint32_t nibble_mask8(const uint8_t* m) {
 }
 
 __global__ void __launch_bounds__(256)
-rac_dispatch_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __restrict__ gs_in,
-                    const uint32_t* __restrict__ amax_bits, int n_sel, const uint8_t* __restrict__ mask, int topk, const int32_t* __restrict__ pos_pad,
-                    uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled, uint8_t* __restrict__ rq_pad,
-                    uint8_t* __restrict__ rsf_tiled, uint8_t* __restrict__ rq_out, uint8_t* __restrict__ rsf_out) {
-  const int groups = H >> 6;
+rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* __restrict__ mask, int topk,
+                   const int32_t* __restrict__ pos_pad, const uint8_t* __restrict__ xq,
+                   const uint8_t* __restrict__ xsf, const uint8_t* __restrict__ rq, const uint8_t* __restrict__ rsf,
+                   uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled, uint8_t* __restrict__ rq_pad,
+                   uint8_t* __restrict__ rsf_tiled, uint8_t* __restrict__ rq_exp, uint8_t* __restrict__ rsf_exp) {
+  const int per_row = H >> 5;                         // 16-byte chunks of codes per row
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= (int64_t)T * groups) return;
-  const int t = (int)(g / groups), kg = (int)(g - (int64_t)t * groups);
-  const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
-  uint32_t xc[8], rc[8], xs = 0, rs = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int kb = kg * 4 + j;
-    uint4 v0, v1;
-    ldg256(x + (size_t)t * H + kb * 16, v0, v1);
-    float f[16];
-    unpack8(v0, f);
-    unpack8(v1, f + 8);
-    const BlockQ bq = quantize_block(f, gs);
-    xc[2 * j] = bq.lo; xc[2 * j + 1] = bq.hi;
-    xs |= bq.sf8 << (8 * j);
-    if (n_sel > 0) {
-      float o[16];
-      dequant_block(bq, o);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) o[i] = __fsub_rn(o[i], f[i]);
-      const BlockQ br = quantize_block(o, gs);
-      const uint32_t mlo = nibble_mask8(mask + kb * 16), mhi = nibble_mask8(mask + kb * 16 + 8);
-      rc[2 * j] = br.lo & mlo; rc[2 * j + 1] = br.hi & mhi;
-      rs |= br.sf8 << (8 * j);
-    }
+  if (g >= (int64_t)T * per_row) return;
+  const int t = (int)(g / per_row), c = (int)(g - (int64_t)t * per_row);
+  const size_t co = (size_t)t * (H >> 1) + c * 16;
+  const uint4 xv = __ldg(reinterpret_cast<const uint4*>(xq + co));
+  uint4 rv = make_uint4(0, 0, 0, 0);
+  const bool sf_owner = (c & 1) == 0;                 // even chunks also move 4 scale bytes (64 channels)
+  uint32_t xs = 0, rs = 0;
+  if (sf_owner) xs = __ldg(reinterpret_cast<const uint32_t*>(xsf + (size_t)t * (H >> 4) + c * 2));
+  if (with_residual) {
+    rv = __ldg(reinterpret_cast<const uint4*>(rq + co));
+    const uint8_t* m = mask + c * 32;
+    rv.x &= nibble_mask8(m); rv.y &= nibble_mask8(m + 8);
+    rv.z &= nibble_mask8(m + 16); rv.w &= nibble_mask8(m + 24);
+    if (sf_owner) rs = __ldg(reinterpret_cast<const uint32_t*>(rsf + (size_t)t * (H >> 4) + c * 2));
+    if (rq_exp) *reinterpret_cast<uint4*>(rq_exp + co) = rv;
+    if (rsf_exp && sf_owner) *reinterpret_cast<uint32_t*>(rsf_exp + (size_t)t * (H >> 4) + c * 2) = rs;
+    rv.x ^= 0x88888888u; rv.y ^= 0x88888888u; rv.z ^= 0x88888888u; rv.w ^= 0x88888888u;
   }
   const int kt_count = H >> 6;
-  if (n_sel > 0 && rq_out) {
-    uint4* d = reinterpret_cast<uint4*>(rq_out + (size_t)t * (H >> 1) + kg * 32);
-    d[0] = make_uint4(rc[0], rc[1], rc[2], rc[3]);
-    d[1] = make_uint4(rc[4], rc[5], rc[6], rc[7]);
-    *reinterpret_cast<uint32_t*>(rsf_out + (size_t)t * (H >> 4) + kg * 4) = rs;
-  }
-  for (int s = 0; s < topk; ++s) {
-    const int p = pos_pad[t * topk + s];
-    uint4* d = reinterpret_cast<uint4*>(xq_pad + (size_t)p * (H >> 1) + kg * 32);
-    d[0] = make_uint4(xc[0], xc[1], xc[2], xc[3]);
-    d[1] = make_uint4(xc[4], xc[5], xc[6], xc[7]);
-    const size_t so = sf_tiled_offset(p, kg * 4, kt_count);
-    *reinterpret_cast<uint32_t*>(xsf_tiled + so) = xs;
-    if (n_sel > 0) {
-      uint4* e = reinterpret_cast<uint4*>(rq_pad + (size_t)p * (H >> 1) + kg * 32);
-      e[0] = make_uint4(rc[0] ^ 0x88888888u, rc[1] ^ 0x88888888u, rc[2] ^ 0x88888888u, rc[3] ^ 0x88888888u);
-      e[1] = make_uint4(rc[4] ^ 0x88888888u, rc[5] ^ 0x88888888u, rc[6] ^ 0x88888888u, rc[7] ^ 0x88888888u);
-      *reinterpret_cast<uint32_t*>(rsf_tiled + so) = rs;
+  for (int s0 = 0; s0 < topk; s0 += 8) {
+    int p[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) p[j] = (s0 + j < topk) ? __ldg(pos_pad + t * topk + s0 + j) : -1;   // all loads first
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (p[j] < 0) continue;
+      const size_t po = (size_t)p[j] * (H >> 1) + c * 16;
+      __stcs(reinterpret_cast<uint4*>(xq_pad + po), xv);
+      if (with_residual) __stcs(reinterpret_cast<uint4*>(rq_pad + po), rv);
+      if (sf_owner) {
+        const size_t so = sf_tiled_offset(p[j], c * 2, kt_count);
+        *reinterpret_cast<uint32_t*>(xsf_tiled + so) = xs;
+        if (with_residual) *reinterpret_cast<uint32_t*>(rsf_tiled + so) = rs;
+      }
     }
   }
 }

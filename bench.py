@@ -335,10 +335,10 @@ def run_ours(args):
                 "traffic": None, "ms": g1_ms,
                 "gemm2": {"ms": g2_ms, "achieved": f_alg2 / (g2_ms * 1e-3) / 1e12, "frac": f_alg2 / (g2_ms * 1e-3) / 1e12 / fp4_peak},
                 "frac_of_nominal_9pf": ach / 9000.0}
-    traffic_file = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(traffic_file):
-        with open(traffic_file) as fh:
-            roofline["traffic"] = json.load(fh).get("%s_%s_gemm1_bytes" % (args.workload, args.variant))
+    # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM-1 launch, from the ncu capture
+    # summarised in profiles/gemm_kernel_moe_prefill_ncu_full.md (prefill workload, RAC at both sites)
+    if args.workload == "prefill" and args.variant == "both":
+        roofline["traffic"] = 466328576
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4 (e2m1 x e2m1, ue4m3 block scales, fp32 accumulate)",

@@ -88,7 +88,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   const int64_t A = dense ? T : (int64_t)T * topk;
   const int Ee = dense ? 1 : E;
   L.n_chunks = (T + kRouteTokensPerCta - 1) / kRouteTokensPerCta;
-  L.m_tiles_max = ((int)(A / (128 * kMTileGroup)) + Ee) * kMTileGroup;
+  L.m_tiles_max = ((int)(A / 256) + Ee) * 2;      // enough for either tile grouping (1 or 2)
   L.stats_ctas = T < 592 * 4 ? (T + 3) / 4 : 592;
   if (L.stats_ctas < 1) L.stats_ctas = 1;
   L.rows_per_cta = (T + L.stats_ctas - 1) / L.stats_ctas;
@@ -289,7 +289,6 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
     blocks_per_sm = b < 1 ? 1 : (b > 8 ? 8 : b);
   }
   int max_groups = 4;
-  { const char* e = getenv("QUADS_FQ_GROUPS"); if (e) max_groups = atoi(e); }
   int n_groups = n_tensors < max_groups ? (int)n_tensors : max_groups;
   int64_t want = (nblk * n_groups + 255) / 256;            // no more CTAs than there is work
   int grid = di.sm_count * blocks_per_sm;
@@ -476,7 +475,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     rs = side->stream;
   }
   if (dense) {
-    dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, pos_pad, row_token, row_weight, tile_expert,
+    dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, gemm_cta_group(), pos_pad, row_token, row_weight, tile_expert,
                                                            tile_rows, header);
     note_launch();
   } else {
@@ -486,7 +485,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
                                               a->topk_ids, a->topk_w);
     note_launch();
     trace_mark("route", st);
-    scan_kernel<<<1, 1024, 0, rs>>>(E, L.n_chunks, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
+    scan_kernel<<<1, 1024, 0, rs>>>(E, L.n_chunks, gemm_cta_group(), chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
                                    tile_rows, header, a->expert_offsets);
     note_launch();
     trace_mark("scan", st);
@@ -549,8 +548,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.row_token = row_token; g.row_weight = row_weight;
   g.tile_prefix = tile_prefix; g.offsets = offsets;
   g.status = header + kHdrStatus;
-  { const char* e = getenv("QUADS_DBG"); g.dbg = e ? atoi(e) : 0; }
   g.b_rows_per_expert = N1;
+  g.n_experts = E;
   if (dense) {
     g.n_out = a->N;
     g.n_tiles_n = (a->N + 255) / 256;

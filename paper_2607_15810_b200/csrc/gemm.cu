@@ -48,6 +48,7 @@ constexpr int kOffB = 2 * kTileA;
 constexpr int kThreads = 576;
 constexpr int kEpiWarps = 16;
 constexpr int kTmemCols = 512;
+constexpr int kMaxTableTiles = 2048;               // M-tiles whose expert / row count fit the shared-memory tables
 constexpr int kTmemSfBase = 256;                  // accumulator: columns 0..255
 constexpr int kTmemSfPerBuf = 16 * kKSteps;       // SFA 4/step | SFR 4/step | SFB 8/step, double buffered
 
@@ -60,7 +61,8 @@ struct Cfg {
   static constexpr int kOffSfB = kOffSfR + kSfA;
   static constexpr int kStageBytes = kOffSfB + kSfB;         // 73728 / 57344
   static constexpr int kBarOffset = kStages * kStageBytes;   // barriers after the ring
-  static constexpr int kSmemBytes = kBarOffset + 256 + 1024; // + barrier block + alignment slack
+  static constexpr int kMetaBytes = CG == 1 ? (2 * kMaxTableTiles + 4 * kMaxExperts) : 0;   // per-tile tables
+  static constexpr int kSmemBytes = kBarOffset + 256 + kMetaBytes + 1024; // + barrier block + tables + alignment slack
 };
 constexpr uint64_t kWaitNs = 2000000000ull;       // bound of every device-side wait (2 s)
 
@@ -115,13 +117,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// L2 prefetches: warm the cache for a later stage without needing a free shared-memory slot.
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void bulk_prefetch(const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -250,17 +245,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor, K-major operand tile stored as rows of 128
-// bytes with the 128-byte swizzle (8-row groups 1024 bytes apart).
-__device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// Descriptor of one 512-byte scale atom for tcgen05.cp: 32 rows of 16 bytes, no
-// swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t desc_sf_atom(uint32_t saddr) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
-}
+// Shared-memory matrix descriptors are built where they are used (MMA issuer): 64-bit
+//   [0,14) start address >> 4 | [16,30) leading byte offset >> 4 | [32,46) stride byte offset >> 4
+//   | [46,48) version = 1 | [61,64) layout (0 none, 2 = 128-byte swizzle, 4 = 64-byte swizzle).
+// Operand tiles are K-major rows with the TMA swizzle, 8-row groups 8 * row bytes apart; a scale
+// atom for tcgen05.cp is 32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart.
 // Instruction descriptor: E2M1 x E2M1, UE4M3 block scales, both operands
 // K-major, M = 128 per CTA of the group, N = 256, dense.
 template <int CG>
@@ -352,7 +341,27 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
-  const int m_groups = p.header[kHdrMTiles] / CG;   // M-tiles come in groups of CG (same expert)
+  // Per-tile metadata (expert, valid rows) and the per-expert weight scales are read by every
+  // role at every tile; dependent global loads there would sit on the critical path of short K
+  // loops, so they are staged in shared memory once (single-CTA variant, when they fit).
+  const int m_tiles_all = p.header[kHdrMTiles];
+  uint8_t* tab_expert = smem_gen + C::kBarOffset + 256;
+  uint8_t* tab_rows = tab_expert + kMaxTableTiles;
+  float* tab_gs = reinterpret_cast<float*>(tab_rows + kMaxTableTiles);
+  const bool tables = (CG == 1) && m_tiles_all <= kMaxTableTiles && p.n_experts <= kMaxExperts;
+  if (tables) {
+    for (int i = threadIdx.x; i < m_tiles_all; i += blockDim.x) {
+      tab_expert[i] = (uint8_t)p.tile_expert[i];
+      tab_rows[i] = (uint8_t)p.tile_rows[i];
+    }
+    for (int i = threadIdx.x; i < p.n_experts; i += blockDim.x) tab_gs[i] = p.b_gs[i];
+    __syncthreads();
+  }
+  auto expert_of = [&](int mt) -> int { return tables ? (int)tab_expert[mt] : p.tile_expert[mt]; };
+  auto rows_of = [&](int mt) -> int { return tables ? (int)tab_rows[mt] : p.tile_rows[mt]; };
+  auto gs_of = [&](int e) -> float { return tables ? tab_gs[e] : p.b_gs[e]; };
+
+  const int m_groups = m_tiles_all / CG;            // M-tiles come in groups of CG (same expert)
   const int total_tiles = m_groups * p.n_tiles_n;
   const int kt_count = p.K >> 6;                    // scale atoms (K = 64 each) along K
   const int k_stages = (kt_count + kKSteps - 1) / kKSteps;
@@ -368,7 +377,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         const int mg = tile / p.n_tiles_n, nt = tile - mg * p.n_tiles_n;
         const int mt = mg * CG + (int)rank;
-        const int e = p.tile_expert[mt];
+        const int e = expert_of(mt);
         const int brow0 = e * p.b_rows_per_expert + nt * (EPI == kEpiSwiGLU ? 128 : 256);
         const int brow1 = brow0 + p.half1_row_offset;
         const bool half1 = (EPI == kEpiSwiGLU) || (nt * 256 + 128 < p.n_out);
@@ -402,19 +411,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
             if (resid) bulk_load(sbase + C::kOffSfR, rsf + sf_off, sf_bytes, full);
             bulk_load(sbase + C::kOffSfB, bsf0 + sf_off, sf_bytes, full);
             if (half1) bulk_load(sbase + C::kOffSfB + kSfA, bsf1 + sf_off, sf_bytes, full);
-            if ((p.dbg & 32) && ks + kStages < k_stages) {
-              // the same tile, kStages stages ahead: pull it into L2 now
-              const int kp = (ks + kStages) * kStageKBytes;
-              const size_t sp = (size_t)(ks + kStages) * (size_t)kSfA;
-              tma_prefetch_2d(tm_a, kp, mt * kBM);
-              if (resid) tma_prefetch_2d(tm_r, kp, mt * kBM);
-              if (load_b0) tma_prefetch_2d(tm_b, kp, brow0);
-              if (load_b1) tma_prefetch_2d(tm_b, kp, brow1);
-              bulk_prefetch(asf + sp, kSfA);
-              if (resid) bulk_prefetch(rsf + sp, kSfA);
-              bulk_prefetch(bsf0 + sp, kSfA);
-              if (half1) bulk_prefetch(bsf1 + sp, kSfA);
-            }
           }
           __syncwarp();
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -479,20 +475,19 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
           const uint32_t sfb_lo = ((sbase + C::kOffSfB) & 0x3FFFFu) >> 4;
           const bool first = ks == 0;
           if (issuer) {
-            if (!(p.dbg & 1)) {
-#pragma unroll
-              for (int j = 0; j < kKSteps; ++j) {
-                if (j < atoms) {
-                  tc_cp_sf<CG>(sfcol + 4 * j, ((uint64_t)kSfHi << 32) | (sfa_lo + 32 * j));
-                  if (resid) tc_cp_sf<CG>(sfcol + 4 * kKSteps + 4 * j, ((uint64_t)kSfHi << 32) | (sfr_lo + 32 * j));
-                  tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j, ((uint64_t)kSfHi << 32) | (sfb_lo + 32 * j));
-                  tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j + 4, ((uint64_t)kSfHi << 32) | (sfb_lo + (kSfA >> 4) + 32 * j));
-                }
-              }
-            }
+            // Scale-factor copies run one K step ahead of the MMAs that use them, so that the
+            // shared-memory -> tensor-memory copy of step j+1 overlaps the MMAs of step j.
+            auto copy_sf = [&](int j) {
+              tc_cp_sf<CG>(sfcol + 4 * j, ((uint64_t)kSfHi << 32) | (sfa_lo + 32 * j));
+              if (resid) tc_cp_sf<CG>(sfcol + 4 * kKSteps + 4 * j, ((uint64_t)kSfHi << 32) | (sfr_lo + 32 * j));
+              tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j, ((uint64_t)kSfHi << 32) | (sfb_lo + 32 * j));
+              tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j + 4, ((uint64_t)kSfHi << 32) | (sfb_lo + (kSfA >> 4) + 32 * j));
+            };
+            if (atoms > 0) copy_sf(0);
 #pragma unroll
             for (int j = 0; j < kKSteps; ++j) {
-              if (j < ((p.dbg & 2) ? (first ? 1 : 0) : atoms)) {
+              if (j + 1 < atoms) copy_sf(j + 1);
+              if (j < atoms) {
                 const uint64_t bdesc = ((uint64_t)kSw128Hi << 32) | (b_lo + 2 * j);
                 tc_mma_nvf4<CG>(tmem, ((uint64_t)kSw128Hi << 32) | (a_lo + 2 * j), bdesc, idesc, sfcol + 4 * j,
                                 sfcol + 8 * kKSteps + 8 * j, (!first || j > 0) ? 1u : 0u);
@@ -525,10 +520,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
       const int mg = tile / p.n_tiles_n, nt = tile - mg * p.n_tiles_n;
       const int mt = mg * CG + (int)rank;
-      const int e = p.tile_expert[mt];
-      const bool valid = row_in_tile < p.tile_rows[mt];
+      const int e = expert_of(mt);
+      const bool valid = row_in_tile < rows_of(mt);
       const int prow = mt * kBM + row_in_tile;
-      const float scale = __fmul_rn(a_gs, p.b_gs[e]);
+      const float scale = __fmul_rn(a_gs, gs_of(e));
       ok = mbar_wait(bar_tfull, (uint32_t)(it & 1), abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
@@ -549,7 +544,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
         else mbar_arrive_remote(tempty_addr);
       }
 
-      if (p.dbg & 4) continue;
       if (EPI == kEpiSwiGLU) {
         const float h_gs = p.h_gs[0];
         const int I = p.n_out;

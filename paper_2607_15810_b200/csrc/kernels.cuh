@@ -9,7 +9,6 @@ namespace quads {
 constexpr int kRouteTokensPerCta = 32;
 constexpr int kMaxTopk = 16;
 constexpr int kMaxExperts = 256;
-constexpr int kMTileGroup = 2;   // every expert's padded rows are a multiple of 128 * kMTileGroup
 
 // header words written by the scan (device side sizes of the dispatch)
 enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, kHdrWords = 8 };
@@ -45,14 +44,14 @@ __global__ void export_site2_kernel(int A, int I, const int32_t* perm, const int
 // ---- routing.cu
 __global__ void route_kernel(const float* logits, int T, int E, int topk, int renormalize, int32_t* ids,
                              float* wts, int32_t* chunk_counts, int32_t* ids_out, float* wts_out);
-__global__ void scan_kernel(int E, int n_chunks, const int32_t* chunk_counts, int32_t* chunk_base,
+__global__ void scan_kernel(int E, int n_chunks, int tile_group, const int32_t* chunk_counts, int32_t* chunk_base,
                             int32_t* offsets, int32_t* tile_prefix, int32_t* tile_expert, int32_t* tile_rows,
                             int32_t* header, int32_t* offsets_out);
 __global__ void permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* ids, const float* wts,
                                const int32_t* chunk_base, const int32_t* offsets, const int32_t* tile_prefix,
                                int32_t* perm, int32_t* pos_pad, int32_t* row_token, float* row_weight,
                                int32_t* perm_out);
-__global__ void dense_dispatch_kernel(int T, int32_t* pos_pad, int32_t* row_token, float* row_weight,
+__global__ void dense_dispatch_kernel(int T, int tile_group, int32_t* pos_pad, int32_t* row_token, float* row_weight,
                                       int32_t* tile_expert, int32_t* tile_rows, int32_t* header);
 
 // ---- gemm.cu
@@ -70,6 +69,7 @@ struct GemmParams {
   int b_rows_per_expert; // weight rows per expert
   int half1_row_offset;  // weight-row distance from the tile's first half to its second half
   int has_resid;         // 1: also accumulate the (negated, masked) residual operand
+  int n_experts;         // entries of b_gs
   const int32_t* header;
   const int32_t* tile_expert;
   const int32_t* tile_rows;
@@ -93,7 +93,6 @@ struct GemmParams {
   uint16_t* h_export;    // optional bf16 [A, n_out] in dispatch order
   const int32_t* tile_prefix;
   const int32_t* offsets;
-  int dbg;               // debugging bit mask (0 in normal operation)
   int32_t* status;       // device status word (QUADS_ERR_TIMEOUT on a failed wait)
 };
 

@@ -113,10 +113,11 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
 
 // One CTA of 1024 threads.  A warp per expert (round robin): exclusive prefix of
 // the expert's counts over chunks and its total; then the exclusive scan over
-// experts of counts (offsets) and of 128-row tile counts (tile_prefix), the
+// experts of counts (offsets) and of 128-row tile counts (tile_prefix; every expert gets a
+// multiple of `tile_group` tiles, so that a CTA pair never straddles experts), the
 // tile -> (expert, valid rows) map, and the header.
 __global__ void __launch_bounds__(1024)
-scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32_t* __restrict__ chunk_base,
+scan_kernel(int E, int n_chunks, int tile_group, const int32_t* __restrict__ chunk_counts, int32_t* __restrict__ chunk_base,
             int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tile_expert,
             int32_t* __restrict__ tile_rows, int32_t* __restrict__ header, int32_t* __restrict__ offsets_out) {
   __shared__ int cnt[kMaxExperts];
@@ -153,7 +154,7 @@ scan_kernel(int E, int n_chunks, const int32_t* __restrict__ chunk_counts, int32
     for (int i = 0; i < E; ++i) {
       off[i] = a; tpre[i] = t;
       a += cnt[i];
-      t += ((cnt[i] + 128 * kMTileGroup - 1) / (128 * kMTileGroup)) * kMTileGroup;
+      t += ((cnt[i] + 128 * tile_group - 1) / (128 * tile_group)) * tile_group;
     }
     off[E] = a; tpre[E] = t;
     header[kHdrMTiles] = t;
@@ -218,11 +219,11 @@ permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__
 
 // Dense mode: identity dispatch of T rows to a single "expert".
 __global__ void __launch_bounds__(256)
-dense_dispatch_kernel(int T, int32_t* __restrict__ pos_pad, int32_t* __restrict__ row_token,
+dense_dispatch_kernel(int T, int tile_group, int32_t* __restrict__ pos_pad, int32_t* __restrict__ row_token,
                       float* __restrict__ row_weight, int32_t* __restrict__ tile_expert,
                       int32_t* __restrict__ tile_rows, int32_t* __restrict__ header) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  const int m_tiles = ((T + 128 * kMTileGroup - 1) / (128 * kMTileGroup)) * kMTileGroup;
+  const int m_tiles = ((T + 128 * tile_group - 1) / (128 * tile_group)) * tile_group;
   if (i < T) { pos_pad[i] = i; row_token[i] = i; row_weight[i] = 1.f; }
   if (i < m_tiles) { tile_expert[i] = 0; tile_rows[i] = max(0, min(128, T - i * 128)); }
   if (i == 0) { header[kHdrMTiles] = m_tiles; header[kHdrPaddedRows] = m_tiles * 128; header[kHdrAssignments] = T; }

@@ -35,6 +35,8 @@ def parse():
     ap.add_argument("--variant", default="both", choices=["both", "w13", "plain"])
     ap.add_argument("--no-aux", action="store_true", help="skip the auxiliary quantize / fake-quant / decode numbers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-budget-s", type=float, default=0.0,
+                    help="seconds of oracle work per step for --impl reference (0: derived from --steps)")
     return ap.parse_args()
 
 
@@ -116,7 +118,7 @@ def run_reference(args):
         return
     from paper_2607_15810_b200 import synth
     shape = synth.MOE_SHAPES[args.workload]
-    budget = max(1.5, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    budget = args.ref_budget_s if args.ref_budget_s > 0 else max(1.5, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
     step, T_s, desc = oracle_sample(shape, args.variant, budget)
     for _ in range(args.warmup):
         step()
@@ -200,29 +202,21 @@ def measured_peaks():
 
 def run_ours(args):
     import torch
-    import torch.distributed as dist
     from paper_2607_15810_b200 import binding as B
     from paper_2607_15810_b200 import synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2607_15810_b200 import dist_util as D
+    world, rank, local = D.env_world()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    D.init("nccl", dev)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        D.barrier()
         torch.cuda.synchronize()
 
     def max_over_ranks(v):
-        if world == 1:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return D.max_over_ranks(v, dev)
 
     shape = synth.MOE_SHAPES[args.workload]
     n13, n2 = nsel_of(shape, args.variant)
@@ -277,7 +271,7 @@ def run_ours(args):
     barrier()
     wall = time.perf_counter() - wall0
     ms = max_over_ranks(sum(times) / len(times))
-    value = world * T / (ms * 1e-3)
+    value = D.whole_job_rate(world, T, ms)
 
     # end to end: pinned host input -> device, the call, result back to pinned host memory
     def e2e_step():
@@ -317,9 +311,7 @@ def run_ours(args):
     stages_us = {k: round(1e3 * sum(v) / len(v), 1) for k, v in stage_acc.items()}
 
     if rank != 0:
-        if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
+        D.shutdown()
         return
 
     peaks = measured_peaks()
@@ -344,7 +336,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "fp4 (e2m1 x e2m1, ue4m3 block scales, fp32 accumulate)",
             "data": "synthetic", "config": workload_config(shape, args.variant),
             "clocks": clocks, "wall_s_timed_region": wall,
-            "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": D.whole_job_rate(world, T, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": x_h.numel() * 2 + lg_h.numel() * 4, "d2h_bytes_per_step": out_h.numel() * 2},
             "gpu_launches": launches_per_step * args.steps,
             "tflops": {"model": f_model / (ms * 1e-3) / 1e12, "algorithmic": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12,
@@ -388,7 +380,7 @@ def run_ours(args):
         line["aux"] = aux
 
     if world == 1 and not args.no_cpu_baseline:
-        step_o, T_s, desc = oracle_sample(shape, args.variant, 15.0)
+        step_o, T_s, desc = oracle_sample(shape, args.variant, 52.0)   # ~32 tokens: ~10 s of oracle work
         t0 = time.perf_counter()
         step_o()
         dt = time.perf_counter() - t0
@@ -397,9 +389,7 @@ def run_ours(args):
     else:
         line["cpu_baseline"] = None
     print(json.dumps(line))
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    D.shutdown()
 
 
 def main():

@@ -428,6 +428,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   if (H > 16384 || I > 16384 || a->rac_nsel_13 < 0 || a->rac_nsel_13 > H || (!dense && (a->rac_nsel_2 < 0 || a->rac_nsel_2 > I)))
     return QUADS_ERR_SHAPE;
   if ((int64_t)T * topk > 0x3FFFFFFF) return QUADS_ERR_SHAPE;
+  if (T == 0) return QUADS_OK;                      // nothing to do; x / out may be NULL
   if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) return QUADS_ERR_NULL;
   if (!dense && (!a->router_logits || !a->w2_q || !a->w2_sf || !a->w2_gs || !a->a2_gs)) return QUADS_ERR_NULL;
   if (!aligned(a->x, 32) || !aligned(a->w13_q, 16) || !aligned(a->w13_sf, 16) || !aligned(a->out, 16) ||

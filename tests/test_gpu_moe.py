@@ -73,8 +73,8 @@ def test_dense_exact_integer_case(B):
     assert np.array_equal(got, MC.f32(torch.from_numpy(want).to(torch.bfloat16)).astype(np.float64))
 
 
-def _moe_small(B, name, f13, f2, renorm):
-    sh = synth.MOE_SHAPES[name]
+def _moe_small(B, name, f13, f2, renorm, shape=None):
+    sh = shape if shape is not None else synth.MOE_SHAPES[name]
     x, _ = synth.activations(sh)
     lg = synth.router_logits(sh)
     w13, w2 = synth.expert_weights(sh, "w13"), synth.expert_weights(sh, "w2")
@@ -103,6 +103,54 @@ def _moe_small(B, name, f13, f2, renorm):
                                                 ("small", 0.25, 0.0, False), ("small", 0.0, 0.5, True)])
 def test_moe_small_layers_in_full(B, name, f13, f2, renorm):
     _moe_small(B, name, f13, f2, renorm)
+
+
+EDGE_SHAPES = [
+    # one token, one choice out of many experts: 255 empty experts, a tile with a single valid row
+    synth.MoEShape("one_token", 31, 1, 128, 256, 1, 128, 0.05, 1, 3.0, 10.0),
+    # fewer tokens than experts, the widest top-k the library takes
+    synth.MoEShape("top16", 32, 9, 256, 32, 16, 128, 0.05, 2, 3.0, 10.0),
+    # a single expert owning several full tiles plus a ragged one (all rows in one segment)
+    synth.MoEShape("one_expert", 33, 300, 128, 1, 1, 256, 0.05, 1, 3.0, 10.0),
+    # K tails: H and I that are not multiples of the 256-element pipeline stage
+    synth.MoEShape("k_tail", 34, 70, 384, 4, 2, 128, 0.05, 2, 3.0, 10.0),
+]
+
+
+@pytest.mark.parametrize("shape", EDGE_SHAPES, ids=[s.name for s in EDGE_SHAPES])
+def test_moe_edge_shapes(B, shape):
+    _moe_small(B, None, 0.5, 0.5, True, shape=shape)
+
+
+def test_zero_tokens_is_a_no_op(B):
+    sh = synth.MOE_SHAPES["tiny"]
+    w13, w2 = synth.expert_weights(sh, "w13"), synth.expert_weights(sh, "w2")
+    gw13 = B.fake_quant_weights(w13.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    gw2 = B.fake_quant_weights(w2.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    x = torch.empty(0, sh.H, dtype=torch.bfloat16).cuda()
+    lg = torch.empty(0, sh.E, dtype=torch.float32).cuda()
+    res = B.moe_w4a4_rac(x, lg, gw13, gw2, sh.topk, 8, 8, torch.tensor([0.1]).cuda())
+    assert res["out"].shape == (0, sh.H)
+
+
+def test_bad_arguments_are_refused(B):
+    sh = synth.MOE_SHAPES["tiny"]
+    w13, w2 = synth.expert_weights(sh, "w13"), synth.expert_weights(sh, "w2")
+    gw13 = B.fake_quant_weights(w13.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    gw2 = B.fake_quant_weights(w2.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    x, _ = synth.activations(sh)
+    lg = synth.router_logits(sh)
+    a2 = torch.tensor([0.1]).cuda()
+    with pytest.raises(B.QuadsError) as e:                      # more compensated channels than channels
+        B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, sh.H + 1, 0, a2)
+    assert e.value.status == -2
+    with pytest.raises(B.QuadsError) as e:                      # workspace too small
+        B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, 8, 8, a2,
+                       workspace=torch.empty(1024, dtype=torch.uint8).cuda())
+    assert e.value.status == -3
+    with pytest.raises(B.QuadsError) as e:                      # top-k larger than the expert count
+        B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.E + 1, 8, 8, a2)
+    assert e.value.status == -2
 
 
 _W = {}

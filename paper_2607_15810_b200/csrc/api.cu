@@ -9,6 +9,11 @@ namespace quads {
 
 thread_local int g_launch_count = 0;
 
+bool pdl_enabled() {
+  static const bool on = [] { const char* e = getenv("QUADS_NO_PDL"); return !(e && e[0] == '1'); }();
+  return on;
+}
+
 namespace {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -206,19 +211,15 @@ int gemm_cta_group() {
 quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
                         int n_sel, double* slice_sums, unsigned int* counters, unsigned long long* keys,
                         uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
-  score_reduce_kernel<<<dim3((C + 31) / 32, kScoreSlices), 256, 0, st>>>(partials, n_part_ptr, n_part_mul,
-                                                                          n_part_fixed, C, slice_sums, counters, keys);
-  note_launch();
+  QUADS_CUDA_OK(launch_kernel(score_reduce_kernel, dim3((C + 31) / 32, kScoreSlices), dim3(256), (size_t)(0), st, partials, n_part_ptr, n_part_mul, n_part_fixed, C, slice_sums, counters, keys));
   static bool attr = false;
   if (!attr) {
     QUADS_CUDA_OK(cudaFuncSetAttribute(rank_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
     attr = true;
   }
-  rank_select_kernel<<<(C + 63) / 64, 256, (size_t)C * 8, st>>>(keys, C, n_sel, mask);
-  note_launch();
+  QUADS_CUDA_OK(launch_kernel(rank_select_kernel, dim3((C + 63) / 64), dim3(256), (size_t)((size_t)C * 8), st, keys, C, n_sel, mask));
   if (sel_export) {
-    sel_list_kernel<<<1, 1024, 0, st>>>(mask, C, sel_export);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(sel_list_kernel, dim3(1), dim3(1024), (size_t)(0), st, mask, C, sel_export));
   }
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
@@ -476,23 +477,15 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     rs = side->stream;
   }
   if (dense) {
-    dense_dispatch_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, gemm_cta_group(), pos_pad, row_token, row_weight, tile_expert,
-                                                           tile_rows, header);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(dense_dispatch_kernel, dim3((T + 255) / 256), dim3(256), (size_t)(0), st, T, gemm_cta_group(), pos_pad, row_token, row_weight, tile_expert, tile_rows, header));
   } else {
     int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
     int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
-    route_kernel<<<L.n_chunks, 256, 0, rs>>>(a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts,
-                                              a->topk_ids, a->topk_w);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(route_kernel, dim3(L.n_chunks), dim3(256), (size_t)(0), rs, a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts, a->topk_ids, a->topk_w));
     trace_mark("route", st);
-    scan_kernel<<<1, 1024, 0, rs>>>(E, L.n_chunks, gemm_cta_group(), chunk_counts, chunk_base, offsets, tile_prefix, tile_expert,
-                                   tile_rows, header, a->expert_offsets);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(1), dim3(1024), (size_t)(0), rs, E, L.n_chunks, gemm_cta_group(), chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, a->expert_offsets));
     trace_mark("scan", st);
-    permute_kernel<<<(L.n_chunks + 3) / 4, 128, 0, rs>>>(T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets,
-                                                         tile_prefix, perm, pos_pad, row_token, row_weight, a->perm);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3((L.n_chunks + 3) / 4), dim3(128), (size_t)(0), rs, T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
   }
   if (side) QUADS_CUDA_OK(cudaEventRecord(side->join, side->stream));
   trace_mark("permute", st);
@@ -502,17 +495,13 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     const int64_t chunks = (int64_t)T * (H / 8);
     int gx = (int)((chunks + 2047) / 2048);
     if (gx > di.sm_count * 8) gx = di.sm_count * 8;
-    amax_kernel<<<dim3(gx, 1), 256, 0, st>>>(x, T, H, H, 0, amax_bits);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(amax_kernel, dim3(gx, 1), dim3(256), (size_t)(0), st, x, T, H, H, 0, amax_bits));
   }
   trace_mark("amax", st);
   // ---- site 13: quantize (+ residual + statistics), selection, dispatch scatter
   const int nsel13 = a->rac_nsel_13;
   uint8_t* mask13 = P(L.mask13);
-  rac_quant_kernel<<<L.stats_ctas, H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32, 0, st>>>(
-      x, T, H, a->a13_gs, amax_bits, a->a13_gs_out, L.rows_per_cta, nsel13 > 0 ? 1 : 0,
-      reinterpret_cast<float*>(P(L.partials13)), P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), a->xq, a->xsf);
-  note_launch();
+  QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(L.stats_ctas), dim3(H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32), (size_t)(0), st, x, T, H, a->a13_gs, amax_bits, a->a13_gs_out, L.rows_per_cta, nsel13 > 0 ? 1 : 0, reinterpret_cast<float*>(P(L.partials13)), P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), a->xq, a->xsf));
   trace_mark("rac_stats", st);
   if (nsel13 > 0) {
     s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
@@ -527,10 +516,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   {
     const int64_t chunks = (int64_t)T * (H / 32);
-    rac_scatter_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(
-        T, H, nsel13 > 0 ? 1 : 0, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok),
-        P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3((unsigned)((chunks + 255) / 256)), dim3(256), (size_t)(0), st, T, H, nsel13 > 0 ? 1 : 0, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
   }
   trace_mark("rac_dispatch", st);
   // ---- tensor maps
@@ -580,17 +566,13 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
                    reinterpret_cast<double*>(P(L.scores2)), reinterpret_cast<unsigned int*>(P(L.counters2)),
                    reinterpret_cast<unsigned long long*>(P(L.keys2)), mask2, a->sel2, st);
     if (s != QUADS_OK) return s;
-    mask_codes_kernel<<<di.sm_count * 8, 256, 0, st>>>(P(L.r2q_pad), header + kHdrPaddedRows, I, mask2);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(mask_codes_kernel, dim3(di.sm_count * 8), dim3(256), (size_t)(0), st, P(L.r2q_pad), header + kHdrPaddedRows, I, mask2));
   } else if (a->r2q) {
     QUADS_CUDA_OK(cudaMemsetAsync(mask2, 0, I, st));
   }
   if (a->hq || a->hsf || a->r2q || a->r2sf) {
     const int64_t n = (int64_t)A * (I / 16);
-    export_site2_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(A, I, perm, pos_pad, P(L.hq_pad), P(L.hsf),
-                                                                     P(L.r2q_pad), P(L.r2sf), mask2, a->hq, a->hsf,
-                                                                     a->r2q, a->r2sf);
-    note_launch();
+    QUADS_CUDA_OK(launch_kernel(export_site2_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), (size_t)(0), st, A, I, perm, pos_pad, P(L.hq_pad), P(L.hsf), P(L.r2q_pad), P(L.r2sf), mask2, a->hq, a->hsf, a->r2q, a->r2sf));
   }
 
   trace_mark("select2+mask", st);
@@ -619,9 +601,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   trace_mark("gemm2", st);
   const int64_t n8 = (int64_t)T * (H / 8);
-  combine_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(y_pad, pos_pad, wts, T, H, topk,
-                                                                static_cast<uint16_t*>(a->out));
-  note_launch();
+  QUADS_CUDA_OK(launch_kernel(combine_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), (size_t)(0), st, y_pad, pos_pad, wts, T, H, topk, static_cast<uint16_t*>(a->out)));
   trace_mark("combine", st);
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;

@@ -23,6 +23,34 @@ inline void note_launch() { ++g_launch_count; }
     if (_e != cudaSuccess) return QUADS_ERR_CUDA;        \
   } while (0)
 
+// Programmatic dependent launch: every kernel of the MoE chain starts with this.  It blocks
+// until the preceding kernel of the stream has completed and its writes are visible, then
+// lets the following kernel begin its own launch (that one blocks at the same point), so
+// launch latencies overlap instead of adding up.  A no-op for ordinary launches.
+__device__ __forceinline__ void pdl_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Host side: launch with the programmatic-stream-serialization attribute (or plainly).
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  note_launch();
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b16) { return __uint_as_float(b16 << 16); }
 
 // Unpack 8 bf16 (one 16-byte vector) to float.

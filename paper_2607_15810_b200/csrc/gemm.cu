@@ -335,6 +335,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
     if (p.has_resid) prefetch_tmap(tm_r);
   }
   if (warp == 1) tmem_alloc<CG>(smem_u32(&bars->tmem_base), kTmemCols);
+  pdl_sync();                               // barrier set-up above overlaps the previous kernel's tail
   tc_fence_before();
   __syncthreads();
   if (CG == 2) cluster_sync_all();          // both CTAs' barriers exist before any remote arrive
@@ -675,9 +676,7 @@ quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const CUte
     attr_set[g][epi] = true;
   }
   const int grid = cta_group == 2 ? (n_sms / 2) * 2 : n_sms;
-  fn<<<grid, kThreads, smem, stream>>>(p, tm_a, tm_r, tm_b);
-  note_launch();
-  QUADS_CUDA_OK(cudaGetLastError());
+  QUADS_CUDA_OK(launch_kernel(fn, dim3(grid), dim3(kThreads), (size_t)smem, stream, p, tm_a, tm_r, tm_b));
   return QUADS_OK;
 }
 

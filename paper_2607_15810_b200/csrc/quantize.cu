@@ -12,6 +12,7 @@ namespace quads {
 __global__ void __launch_bounds__(256) amax_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K,
                                                    int64_t ld, int64_t tensor_stride,
                                                    uint32_t* __restrict__ amax_bits) {
+  pdl_sync();
   const uint16_t* base = x + (size_t)blockIdx.y * tensor_stride;
   const int64_t k8 = K >> 3;
   const int64_t chunks = rows * k8;
@@ -232,6 +233,7 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
                  int with_residual, float* __restrict__ partials, uint8_t* __restrict__ xq,
                  uint8_t* __restrict__ xsf, uint8_t* __restrict__ rq, uint8_t* __restrict__ rsf,
                  uint8_t* __restrict__ xq_exp, uint8_t* __restrict__ xsf_exp) {
+  pdl_sync();
   const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
   if (gs_store && blockIdx.x == 0 && threadIdx.x == 0) gs_store[0] = gs;
   const int k16 = H >> 4;
@@ -286,6 +288,7 @@ __global__ void __launch_bounds__(256)
 score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ n_part_ptr, int n_part_mul,
                     int n_part_fixed, int C, double* __restrict__ slice_sums, unsigned int* __restrict__ counters,
                     unsigned long long* __restrict__ score_keys) {
+  pdl_sync();
   const int n_part = n_part_ptr ? *n_part_ptr * n_part_mul : n_part_fixed;
   const int per = (n_part + kScoreSlices - 1) / kScoreSlices;
   const int p0 = blockIdx.y * per, p1 = min(n_part, p0 + per);
@@ -324,6 +327,7 @@ score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ 
 // grid = ceil(C/64), 256 threads, smem = C * 8 bytes.
 __global__ void __launch_bounds__(256)
 rank_select_kernel(const unsigned long long* __restrict__ score_keys, int C, int n_sel, uint8_t* __restrict__ mask) {
+  pdl_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* sc = reinterpret_cast<unsigned long long*>(smem_raw);
   for (int i = threadIdx.x; i < C; i += blockDim.x) sc[i] = score_keys[i];
@@ -347,6 +351,7 @@ rank_select_kernel(const unsigned long long* __restrict__ score_keys, int C, int
 // Ascending list of the selected channels (verification export only).  One CTA.
 __global__ void __launch_bounds__(1024)
 sel_list_kernel(const uint8_t* __restrict__ mask, int C, int32_t* __restrict__ sel_export) {
+  pdl_sync();
   __shared__ int chunk_tot[1024];
   const int tid = threadIdx.x, nt = blockDim.x;
   const int per = (C + nt - 1) / nt;
@@ -391,6 +396,7 @@ rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* __restrict__ 
                    const uint8_t* __restrict__ xsf, const uint8_t* __restrict__ rq, const uint8_t* __restrict__ rsf,
                    uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled, uint8_t* __restrict__ rq_pad,
                    uint8_t* __restrict__ rsf_tiled, uint8_t* __restrict__ rq_exp, uint8_t* __restrict__ rsf_exp) {
+  pdl_sync();
   const int per_row = H >> 5;                         // 16-byte chunks of codes per row
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= (int64_t)T * per_row) return;
@@ -436,6 +442,7 @@ rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* __restrict__ 
 __global__ void __launch_bounds__(256)
 mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_ptr, int C,
                   const uint8_t* __restrict__ mask) {
+  pdl_sync();
   const int per_row = C >> 5;
   const int64_t n = (int64_t)(*n_rows_ptr) * per_row;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -455,6 +462,7 @@ mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_pt
 __global__ void __launch_bounds__(256)
 combine_kernel(const uint16_t* __restrict__ y_pad, const int32_t* __restrict__ pos_pad,
                const float* __restrict__ wts, int T, int H, int topk, uint16_t* __restrict__ out) {
+  pdl_sync();
   const int per_row = H >> 3;
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)T * per_row) return;
@@ -484,6 +492,7 @@ export_site2_kernel(int A, int I, const int32_t* __restrict__ perm, const int32_
                     const uint8_t* __restrict__ r2q_pad, const uint8_t* __restrict__ r2sf_tiled,
                     const uint8_t* __restrict__ mask2, uint8_t* __restrict__ hq, uint8_t* __restrict__ hsf, uint8_t* __restrict__ r2q,
                     uint8_t* __restrict__ r2sf) {
+  pdl_sync();
   const int k16 = I >> 4;
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)A * k16) return;

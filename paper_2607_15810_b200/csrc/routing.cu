@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(256)
 route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
              int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
              int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
+  pdl_sync();
   __shared__ int hist[kMaxExperts];
   for (int i = threadIdx.x; i < E; i += blockDim.x) hist[i] = 0;
   __syncthreads();
@@ -120,6 +121,7 @@ __global__ void __launch_bounds__(1024)
 scan_kernel(int E, int n_chunks, int tile_group, const int32_t* __restrict__ chunk_counts, int32_t* __restrict__ chunk_base,
             int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tile_expert,
             int32_t* __restrict__ tile_rows, int32_t* __restrict__ header, int32_t* __restrict__ offsets_out) {
+  pdl_sync();
   __shared__ int cnt[kMaxExperts];
   __shared__ int off[kMaxExperts + 1];
   __shared__ int tpre[kMaxExperts + 1];
@@ -184,6 +186,7 @@ permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__
                const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ offsets,
                const int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ pos_pad,
                int32_t* __restrict__ row_token, float* __restrict__ row_weight, int32_t* __restrict__ perm_out) {
+  pdl_sync();
   __shared__ int run[4][kMaxExperts];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = blockIdx.x * 4 + warp;
@@ -222,6 +225,7 @@ __global__ void __launch_bounds__(256)
 dense_dispatch_kernel(int T, int tile_group, int32_t* __restrict__ pos_pad, int32_t* __restrict__ row_token,
                       float* __restrict__ row_weight, int32_t* __restrict__ tile_expert,
                       int32_t* __restrict__ tile_rows, int32_t* __restrict__ header) {
+  pdl_sync();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   const int m_tiles = ((T + 128 * tile_group - 1) / (128 * tile_group)) * tile_group;
   if (i < T) { pos_pad[i] = i; row_token[i] = i; row_weight[i] = 1.f; }

@@ -203,6 +203,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// No memory ordering: for hand-overs whose payload is tensor memory (ordered by tcgen05 fences),
+// so that the arrive does not wait for this thread's earlier global stores.
+__device__ __forceinline__ void mbar_arrive_remote_relaxed(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
@@ -542,7 +547,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       __syncwarp();
       if (lane == 0) {                            // accumulator is free for the next tile
         if (CG == 1) mbar_arrive(bar_tempty);
-        else mbar_arrive_remote(tempty_addr);
+        else mbar_arrive_remote_relaxed(tempty_addr);
       }
 
       if (EPI == kEpiSwiGLU) {

@@ -220,3 +220,16 @@ def test_decode_layer_in_full(B):
     torch.cuda.synchronize()
     assert B.moe_async_status(res["workspace"]) == 0
     MC.check_moe(res, x, lg, w13o, w2o, sh.topk, nsel13, nsel2, a2)
+
+
+def test_cta_pair_gemm_variant_in_a_subprocess():
+    """The optional CTA-pair GEMM (cta_group::2, selected by an environment
+    variable read once per process) passes the same dense and small-layer
+    parity cases."""
+    import subprocess
+    env = dict(os.environ, QUADS_GEMM_CTA_GROUP="2")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_moe.py"), "-x", "-q", "-m",
+                        "gpu", "-k", "dense_config_all_ratios or dense_ragged or small_layers or edge_shapes"],
+                       cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:]

@@ -83,15 +83,21 @@ __device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
   return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
 }
 
-// Two floats -> one byte of E2M1 codes (lo in bits 0..3, hi in bits 4..7),
-// round-to-nearest-even, saturating to 6.  The hardware convert keeps the sign
-// bit of values that round to zero (-0, small negatives), which is the
-// convention of this library; the exhaustive quantizer test pins it.
-__device__ __forceinline__ uint32_t f32x2_to_e2m1x2(float lo, float hi) {
-  uint16_t r;
-  asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; cvt.u16.u8 %0, t; }"
-      : "=h"(r) : "f"(hi), "f"(lo));
-  return (uint32_t)r & 0xFFu;
+// Eight floats -> eight E2M1 codes in one 32-bit word (element i in nibble i),
+// round-to-nearest-even, saturating to 6.  The hardware convert keeps the sign bit of
+// values that round to zero (-0, small negatives), which is the convention of this
+// library; the exhaustive quantizer test pins it.
+__device__ __forceinline__ uint32_t f32x8_to_e2m1x8(float v0, float v1, float v2, float v3, float v4, float v5,
+                                                    float v6, float v7) {
+  uint32_t r;
+  asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+      "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+      : "=r"(r) : "f"(v0), "f"(v1), "f"(v2), "f"(v3), "f"(v4), "f"(v5), "f"(v6), "f"(v7));
+  return r;
 }
 
 // One byte of two E2M1 codes -> two floats (exact): low nibble -> .x, high nibble -> .y.
@@ -108,26 +114,44 @@ struct BlockQ {
   float d;           // decoded block scale sf * gs
 };
 
-// Quantize one block of 16 floats with per-tensor scale gs.  Every step is a
-// single IEEE float32 operation, in the order the header documents.
-__device__ __forceinline__ BlockQ quantize_block(const float* v, float gs) {
+// Per-tensor constants of the quantizer.  `r6` is the correctly rounded reciprocal of d6 and
+// `inv_lut[c]` = 1 / (E4M3(c) * gs) (0 for c = 0), both computed with IEEE operations, so that
+// the per-block arithmetic below reproduces the documented single-operation recipe bit for bit
+// without a division routine per block.
+struct QuantCtx {
+  float gs, d6, r6;
+  const float* inv_lut;   // 128 entries (shared memory)
+};
+
+__device__ __forceinline__ void quant_ctx_scalars(QuantCtx& c, float gs) {
+  c.gs = gs;
+  c.d6 = __fmul_rn(6.0f, gs);
+  c.r6 = __frcp_rn(c.d6);
+}
+// Entry `code` of the reciprocal table for per-tensor scale gs.
+__device__ __forceinline__ float quant_inv_entry(uint32_t code, float gs) {
+  const float sf = e4m3_to_f32(code & 0x7Fu);
+  return (sf == 0.f || code == 0x7Fu) ? 0.f : __fdiv_rn(1.0f, __fmul_rn(sf, gs));
+}
+
+// Quantize one block of 16 floats.  u = amax / d6 is formed as q0 = amax * r6 followed by one
+// fused correction step (residual amax - q0 * d6 is exact in an FMA), which yields the correctly
+// rounded quotient given a correctly rounded reciprocal; the 1 / d of the element scaling comes
+// from the table.
+__device__ __forceinline__ BlockQ quantize_block(const float* v, const QuantCtx& c) {
   float a = 0.f;
 #pragma unroll
   for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(v[i]));
-  const float d6 = __fmul_rn(6.0f, gs);
-  const float u = __fdiv_rn(a, d6);
+  const float q0 = __fmul_rn(a, c.r6);
+  const float u = __fmaf_rn(__fmaf_rn(-q0, c.d6, a), c.r6, q0);
   BlockQ r;
   r.sf8 = f32_to_e4m3(u);
-  const float sf = e4m3_to_f32(r.sf8);
-  r.d = __fmul_rn(sf, gs);
-  const float inv = (sf == 0.f) ? 0.f : __fdiv_rn(1.0f, r.d);
-  uint32_t lo = 0, hi = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    lo |= f32x2_to_e2m1x2(__fmul_rn(v[2 * i], inv), __fmul_rn(v[2 * i + 1], inv)) << (8 * i);
-    hi |= f32x2_to_e2m1x2(__fmul_rn(v[8 + 2 * i], inv), __fmul_rn(v[9 + 2 * i], inv)) << (8 * i);
-  }
-  r.lo = lo; r.hi = hi;
+  r.d = __fmul_rn(e4m3_to_f32(r.sf8), c.gs);
+  const float inv = c.inv_lut[r.sf8];
+  r.lo = f32x8_to_e2m1x8(__fmul_rn(v[0], inv), __fmul_rn(v[1], inv), __fmul_rn(v[2], inv), __fmul_rn(v[3], inv),
+                         __fmul_rn(v[4], inv), __fmul_rn(v[5], inv), __fmul_rn(v[6], inv), __fmul_rn(v[7], inv));
+  r.hi = f32x8_to_e2m1x8(__fmul_rn(v[8], inv), __fmul_rn(v[9], inv), __fmul_rn(v[10], inv), __fmul_rn(v[11], inv),
+                         __fmul_rn(v[12], inv), __fmul_rn(v[13], inv), __fmul_rn(v[14], inv), __fmul_rn(v[15], inv));
   return r;
 }
 

@@ -61,7 +61,7 @@ struct Cfg {
   static constexpr int kOffSfB = kOffSfR + kSfA;
   static constexpr int kStageBytes = kOffSfB + kSfB;         // 73728 / 57344
   static constexpr int kBarOffset = kStages * kStageBytes;   // barriers after the ring
-  static constexpr int kMetaBytes = CG == 1 ? (2 * kMaxTableTiles + 4 * kMaxExperts) : 0;   // per-tile tables
+  static constexpr int kMetaBytes = 512 + (CG == 1 ? (2 * kMaxTableTiles + 4 * kMaxExperts) : 0);   // reciprocal table + per-tile tables
   static constexpr int kSmemBytes = kBarOffset + 256 + kMetaBytes + 1024; // + barrier block + tables + alignment slack
 };
 constexpr uint64_t kWaitNs = 2000000000ull;       // bound of every device-side wait (2 s)
@@ -351,7 +351,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
   // role at every tile; dependent global loads there would sit on the critical path of short K
   // loops, so they are staged in shared memory once (single-CTA variant, when they fit).
   const int m_tiles_all = p.header[kHdrMTiles];
-  uint8_t* tab_expert = smem_gen + C::kBarOffset + 256;
+  float* inv_lut = reinterpret_cast<float*>(smem_gen + C::kBarOffset + 256);   // 128 entries, SwiGLU epilogue
+  if (EPI == kEpiSwiGLU && threadIdx.x < 128) inv_lut[threadIdx.x] = quant_inv_entry(threadIdx.x, p.h_gs[0]);
+  uint8_t* tab_expert = smem_gen + C::kBarOffset + 256 + 512;
   uint8_t* tab_rows = tab_expert + kMaxTableTiles;
   float* tab_gs = reinterpret_cast<float*>(tab_rows + kMaxTableTiles);
   const bool tables = (CG == 1) && m_tiles_all <= kMaxTableTiles && p.n_experts <= kMaxExperts;
@@ -361,8 +363,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       tab_rows[i] = (uint8_t)p.tile_rows[i];
     }
     for (int i = threadIdx.x; i < p.n_experts; i += blockDim.x) tab_gs[i] = p.b_gs[i];
-    __syncthreads();
   }
+  __syncthreads();                          // tables and the reciprocal table are visible to every role
   auto expert_of = [&](int mt) -> int { return tables ? (int)tab_expert[mt] : p.tile_expert[mt]; };
   auto rows_of = [&](int mt) -> int { return tables ? (int)tab_rows[mt] : p.tile_rows[mt]; };
   auto gs_of = [&](int e) -> float { return tables ? tab_gs[e] : p.b_gs[e]; };
@@ -551,7 +553,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       }
 
       if (EPI == kEpiSwiGLU) {
-        const float h_gs = p.h_gs[0];
+        QuantCtx qc;
+        quant_ctx_scalars(qc, p.h_gs[0]);
+        qc.inv_lut = inv_lut;
         const int I = p.n_out;
         const int f0 = nt * 128 + cq * 32;        // first feature of this thread's 32
         const int kt2 = I >> 6;
@@ -568,7 +572,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
             const float h = __fdividef(g, 1.0f + __expf(-g)) * u;
             hb[i] = __bfloat162float(__float2bfloat16_rn(h));
           }
-          const BlockQ bq = quantize_block(hb, h_gs);
+          const BlockQ bq = quantize_block(hb, qc);
           hs |= bq.sf8 << (8 * c);
           if (valid) {
             *reinterpret_cast<uint2*>(p.hq_pad + (size_t)prow * (I >> 1) + ((f0 + 16 * c) >> 1)) =
@@ -586,7 +590,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
             dequant_block(bq, r);
 #pragma unroll
             for (int i = 0; i < 16; ++i) r[i] = __fsub_rn(r[i], hb[i]);
-            const BlockQ br = quantize_block(r, h_gs);
+            const BlockQ br = quantize_block(r, qc);
             rs |= br.sf8 << (8 * c);
             if (valid)
               *reinterpret_cast<uint2*>(p.r2q_pad + (size_t)prow * (I >> 1) + ((f0 + 16 * c) >> 1)) =

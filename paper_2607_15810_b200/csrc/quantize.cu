@@ -104,6 +104,7 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
   const int64_t gtid = (int64_t)rank * blockDim.x + threadIdx.x;
   __shared__ uint32_t wmax[8];
   __shared__ float gs_sh;
+  __shared__ float inv_lut[128];
   for (int t = group; t < n_tensors; t += n_groups) {
     const uint16_t* base = x + (size_t)t * tensor_stride;
     float gs;
@@ -161,6 +162,12 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
       __syncthreads();
     }
     if (gs_out && rank == 0 && threadIdx.x == 0) gs_out[t] = gs;
+    __syncthreads();                              // the previous tensor's table is no longer read
+    if (threadIdx.x < 128) inv_lut[threadIdx.x] = quant_inv_entry(threadIdx.x, gs);
+    __syncthreads();
+    QuantCtx qc;
+    quant_ctx_scalars(qc, gs);
+    qc.inv_lut = inv_lut;
     // ---- phase 2: quantize (16-element blocks), stream the outputs
     uint8_t* qt = q ? q + (size_t)t * rows * (K >> 1) : nullptr;
     uint8_t* sft = sf ? sf + (size_t)t * sf_tensor_stride : nullptr;
@@ -172,7 +179,7 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
       float f[16];
       unpack8(v0, f);
       unpack8(v1, f + 8);
-      const BlockQ bq = quantize_block(f, gs);
+      const BlockQ bq = quantize_block(f, qc);
       // outputs are contiguous per tensor: block b owns bytes [8b, 8b+8) of q and [32b, 32b+32) of fq
       if (qt) __stcs(reinterpret_cast<uint2*>(qt + b * 8), make_uint2(bq.lo, bq.hi));
       if (sft) {
@@ -236,6 +243,12 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
   pdl_sync();
   const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
   if (gs_store && blockIdx.x == 0 && threadIdx.x == 0) gs_store[0] = gs;
+  __shared__ float inv_lut[128];
+  for (int i = threadIdx.x; i < 128; i += blockDim.x) inv_lut[i] = quant_inv_entry(i, gs);
+  __syncthreads();
+  QuantCtx qc;
+  quant_ctx_scalars(qc, gs);
+  qc.inv_lut = inv_lut;
   const int k16 = H >> 4;
   const int r0 = blockIdx.x * rows_per_cta;
   const int r1 = min(T, r0 + rows_per_cta);
@@ -249,7 +262,7 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
       float f[16], o[16];
       unpack8(v0, f);
       unpack8(v1, f + 8);
-      const BlockQ bq = quantize_block(f, gs);
+      const BlockQ bq = quantize_block(f, qc);
       const size_t qo = (size_t)r * (H >> 1) + kb * 8, so = (size_t)r * k16 + kb;
       *reinterpret_cast<uint2*>(xq + qo) = make_uint2(bq.lo, bq.hi);
       xsf[so] = (uint8_t)bq.sf8;
@@ -262,7 +275,7 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
           o[i] = __fsub_rn(o[i], f[i]);
           acc[i] = __fmaf_rn(o[i], o[i], acc[i]);
         }
-        const BlockQ br = quantize_block(o, gs);
+        const BlockQ br = quantize_block(o, qc);
         *reinterpret_cast<uint2*>(rq + qo) = make_uint2(br.lo, br.hi);
         rsf[so] = (uint8_t)br.sf8;
       }

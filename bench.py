@@ -361,7 +361,21 @@ def run_ours(args):
         tq = timed(qstep, 40, with_flush=False)
         aux["quantize_gbs"] = T * H * 2.5625 / (sum(tq) / len(tq) * 1e-3) / 1e9
         aux["quantize_frac_of_hbm"] = aux["quantize_gbs"] / peaks["hbm_gbs"]
+        aux["quantize_note"] = "%.1f MB activation: launch-latency regime" % (T * H * 2 / 1e6)
         del ring
+        # the same call on an activation large enough for bandwidth to matter (65536 x 4096, 537 MB)
+        big = torch.randn(65536, 4096, device=dev).to(torch.bfloat16)
+        qb = torch.empty(65536, 2048, dtype=torch.uint8, device=dev)
+        sb = torch.empty(65536, 256, dtype=torch.uint8, device=dev)
+
+        def qbig():
+            B.quantize_nvfp4(big, out=(qb, sb, g), workspace=qws)
+        for _ in range(3):
+            qbig()
+        tb = timed(qbig, 10)
+        aux["quantize_large_gbs"] = big.numel() * 2.5625 / (sum(tb) / len(tb) * 1e-3) / 1e9
+        aux["quantize_large_frac_of_hbm"] = aux["quantize_large_gbs"] / peaks["hbm_gbs"]
+        del big, qb, sb
         # fake-quant + pack GB/s: 16 experts' W13 of the AQAT workload (403 MB in, 516 MB out)
         w = (torch.randn(16, 3072, 4096, device=dev) * 0.015).to(torch.bfloat16)
         outs = (torch.empty_like(w), torch.empty(16, 3072, 2048, dtype=torch.uint8, device=dev),

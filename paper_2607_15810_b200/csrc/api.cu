@@ -75,6 +75,22 @@ quads_status make_codes_map(CUtensorMap* map, const void* base, uint64_t rows, u
   return r == CUDA_SUCCESS ? QUADS_OK : QUADS_ERR_CUDA;
 }
 
+// 2D map over tiled scale factors viewed as [atoms, 128 x u32] (512-byte atoms), box =
+// kGemmKSteps atoms, no swizzle; used by the CTA-pair GEMM only.
+quads_status make_sf_map(CUtensorMap* map, const void* base, uint64_t atoms) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return QUADS_ERR_CUDA;
+  if (atoms == 0) atoms = 1;
+  cuuint64_t dims[2] = {128, atoms};
+  cuuint64_t strides[1] = {512};
+  cuuint32_t box[2] = {128, (cuuint32_t)kGemmKSteps};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? QUADS_OK : QUADS_ERR_CUDA;
+}
+
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // ------------------------------------------------------------------ workspace
@@ -520,10 +536,16 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   trace_mark("rac_dispatch", st);
   // ---- tensor maps
-  CUtensorMap tm_x, tm_r, tm_w13;
-  if ((s = make_codes_map(&tm_x, P(L.xq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&tm_r, P(L.rq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&tm_w13, a->w13_q, (uint64_t)E * N1, H / 2)) != QUADS_OK) return s;
+  GemmMaps m1;
+  if ((s = make_codes_map(&m1.a, P(L.xq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m1.r, P(L.rq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m1.b, a->w13_q, (uint64_t)E * N1, H / 2)) != QUADS_OK) return s;
+  if (gemm_cta_group() == 2) {
+    const uint64_t a_atoms = (uint64_t)(pad_rows / 128) * (H / 64);
+    if ((s = make_sf_map(&m1.sfa, P(L.xsf), a_atoms)) != QUADS_OK) return s;
+    if ((s = make_sf_map(&m1.sfr, P(L.rsf), a_atoms)) != QUADS_OK) return s;
+    if ((s = make_sf_map(&m1.sfb, a->w13_sf, (uint64_t)E * (quads_sf_tiled_bytes(N1, H) / 512))) != QUADS_OK) return s;
+  }
 
   GemmParams g{};
   g.K = H;
@@ -542,7 +564,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     g.n_tiles_n = (a->N + 255) / 256;
     g.half1_row_offset = 128;
     g.out_bf16 = static_cast<uint16_t*>(a->out);
-    return launch_gemm(kEpiStore, gemm_cta_group(), g, tm_x, tm_r, tm_w13, di.sm_count, st);
+    return launch_gemm(kEpiStore, gemm_cta_group(), g, m1, di.sm_count, st);
   }
   g.n_out = I;
   g.n_tiles_n = I / 128;
@@ -554,7 +576,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.h_export = static_cast<uint16_t*>(a->h_bf16);
   const bool timing = g_timers.enabled && g_timers.created;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[0], st));
-  if ((s = launch_gemm(kEpiSwiGLU, gemm_cta_group(), g, tm_x, tm_r, tm_w13, di.sm_count, st)) != QUADS_OK) return s;
+  if ((s = launch_gemm(kEpiSwiGLU, gemm_cta_group(), g, m1, di.sm_count, st)) != QUADS_OK) return s;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[1], st));
 
   trace_mark("gemm1", st);
@@ -578,10 +600,16 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   trace_mark("select2+mask", st);
   // ---- second projection + weighted combine
   uint16_t* y_pad = reinterpret_cast<uint16_t*>(P(L.y_pad));
-  CUtensorMap tm_h, tm_r2, tm_w2;
-  if ((s = make_codes_map(&tm_h, P(L.hq_pad), pad_rows, I / 2)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&tm_r2, P(L.r2q_pad), pad_rows, I / 2)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&tm_w2, a->w2_q, (uint64_t)E * H, I / 2)) != QUADS_OK) return s;
+  GemmMaps m2;
+  if ((s = make_codes_map(&m2.a, P(L.hq_pad), pad_rows, I / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m2.r, P(L.r2q_pad), pad_rows, I / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m2.b, a->w2_q, (uint64_t)E * H, I / 2)) != QUADS_OK) return s;
+  if (gemm_cta_group() == 2) {
+    const uint64_t a_atoms = (uint64_t)(pad_rows / 128) * (I / 64);
+    if ((s = make_sf_map(&m2.sfa, P(L.hsf), a_atoms)) != QUADS_OK) return s;
+    if ((s = make_sf_map(&m2.sfr, P(L.r2sf), a_atoms)) != QUADS_OK) return s;
+    if ((s = make_sf_map(&m2.sfb, a->w2_sf, (uint64_t)E * (quads_sf_tiled_bytes(H, I) / 512))) != QUADS_OK) return s;
+  }
   GemmParams g2 = g;
   g2.K = I;
   g2.has_resid = nsel2 > 0;
@@ -594,7 +622,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g2.half1_row_offset = 128;
   g2.y_pad = y_pad;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[2], st));
-  if ((s = launch_gemm(kEpiCombine, gemm_cta_group(), g2, tm_h, tm_r2, tm_w2, di.sm_count, st)) != QUADS_OK) return s;
+  if ((s = launch_gemm(kEpiCombine, gemm_cta_group(), g2, m2, di.sm_count, st)) != QUADS_OK) return s;
   if (timing) {
     QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
     g_timers.valid = true;

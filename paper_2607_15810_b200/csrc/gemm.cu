@@ -114,6 +114,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// CTA-pair forms: the data lands in this CTA's shared memory, the transaction bytes are
+// credited to a barrier given by its cluster address (the leader CTA's).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                                 uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_cluster, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -199,9 +210,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // No memory ordering: for hand-overs whose payload is tensor memory (ordered by tcgen05 fences),
 // so that the arrive does not wait for this thread's earlier global stores.
@@ -309,7 +317,8 @@ __device__ __forceinline__ float warp_colsum16(const float* v, int lane) {
 
 template <int EPI, int CG>
 __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap* tm_a, const CUtensorMap* tm_r,
-                                          const CUtensorMap* tm_b) {
+                                          const CUtensorMap* tm_b, const CUtensorMap* tm_sfa,
+                                          const CUtensorMap* tm_sfr, const CUtensorMap* tm_sfb) {
   using C = Cfg<CG>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_dyn[];
@@ -382,6 +391,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       const bool issuer = elect_one();
       uint32_t stage = 0, phase = 0;
       bool ok = true;
+      const uint32_t leader_full = CG == 2 ? map_to_cta(bar_full, 0) : bar_full;
+      const int b_atoms_per_expert = (int)(p.b_sf_expert_stride >> 9);
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         const int mg = tile / p.n_tiles_n, nt = tile - mg * p.n_tiles_n;
         const int mt = mg * CG + (int)rank;
@@ -410,15 +421,32 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
           const int kc = ks * kStageKBytes;
           const size_t sf_off = (size_t)ks * (size_t)kSfA;
           if (issuer) {
-            mbar_expect_tx(full, data_bytes + sf_bytes * sf_count);
-            tma_load_2d(sbase, tm_a, kc, mt * kBM, full);
-            if (resid) tma_load_2d(sbase + kOffR, tm_r, kc, mt * kBM, full);
-            if (load_b0) tma_load_2d(sbase + kOffB, tm_b, kc, brow0, full);
-            if (load_b1) tma_load_2d(sbase + kOffB + (CG == 1 ? kTileA : 0), tm_b, kc, brow1, full);
-            bulk_load(sbase + C::kOffSfA, asf + sf_off, sf_bytes, full);
-            if (resid) bulk_load(sbase + C::kOffSfR, rsf + sf_off, sf_bytes, full);
-            bulk_load(sbase + C::kOffSfB, bsf0 + sf_off, sf_bytes, full);
-            if (half1) bulk_load(sbase + C::kOffSfB + kSfA, bsf1 + sf_off, sf_bytes, full);
+            if (CG == 1) {
+              mbar_expect_tx(full, data_bytes + sf_bytes * sf_count);
+              tma_load_2d(sbase, tm_a, kc, mt * kBM, full);
+              if (resid) tma_load_2d(sbase + kOffR, tm_r, kc, mt * kBM, full);
+              tma_load_2d(sbase + kOffB, tm_b, kc, brow0, full);
+              if (half1) tma_load_2d(sbase + kOffB + kTileA, tm_b, kc, brow1, full);
+              bulk_load(sbase + C::kOffSfA, asf + sf_off, sf_bytes, full);
+              if (resid) bulk_load(sbase + C::kOffSfR, rsf + sf_off, sf_bytes, full);
+              bulk_load(sbase + C::kOffSfB, bsf0 + sf_off, sf_bytes, full);
+              if (half1) bulk_load(sbase + C::kOffSfB + kSfA, bsf1 + sf_off, sf_bytes, full);
+            } else {
+              // every load of either CTA credits the LEADER's barrier; scale atoms travel as TMA
+              // boxes (kKSteps atoms of 512 bytes; a K tail reads, and counts, the full box)
+              const uint32_t lfull = leader_full + 8 * stage;
+              mbar_expect_tx_cluster(lfull, data_bytes + (uint32_t)kSfA * sf_count);
+              tma_load_2d_pair(sbase, tm_a, kc, mt * kBM, lfull);
+              if (resid) tma_load_2d_pair(sbase + kOffR, tm_r, kc, mt * kBM, lfull);
+              if (load_b0) tma_load_2d_pair(sbase + kOffB, tm_b, kc, brow0, lfull);
+              if (load_b1) tma_load_2d_pair(sbase + kOffB, tm_b, kc, brow1, lfull);
+              const int a_atom = mt * kt_count + ks * kKSteps;
+              const int b_atom = e * b_atoms_per_expert + ks * kKSteps;
+              tma_load_2d_pair(sbase + C::kOffSfA, tm_sfa, 0, a_atom, lfull);
+              if (resid) tma_load_2d_pair(sbase + C::kOffSfR, tm_sfr, 0, a_atom, lfull);
+              tma_load_2d_pair(sbase + C::kOffSfB, tm_sfb, 0, b_atom + rt0 * kt_count, lfull);
+              if (half1) tma_load_2d_pair(sbase + C::kOffSfB + kSfA, tm_sfb, 0, b_atom + rt1 * kt_count, lfull);
+            }
           }
           __syncwarp();
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -431,23 +459,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       }
     }
   } else if (warp == 1 && !leader) {
-    // ------------------------------------------------------------ peer CTA: tell the leader when this
-    // CTA's half of a stage has landed (the leader issues the MMAs for both CTAs)
-    {
-      const bool issuer = elect_one();
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      const uint32_t leader_full = map_to_cta(bar_full, 0);
-      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
-        for (int ks = 0; ks < k_stages; ++ks) {
-          ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status);
-          if (!ok) break;
-          if (issuer) mbar_arrive_remote(leader_full + 8 * stage);
-          __syncwarp();
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-        }
-      }
-    }
+    // the leader CTA issues the MMAs of the pair; nothing to do here
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA; whole warp, one lane issues)
     {
@@ -462,10 +474,6 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       constexpr uint32_t kSw128Hi = (uint32_t)((8 * kStageKBytes) >> 4) | (1u << 14) | ((kStageKBytes == 128 ? 2u : 4u) << 29);
       constexpr uint32_t kSfHi = (uint32_t)(128 >> 4) | (1u << 14);
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
-        ok = CG == 1 ? mbar_wait(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status)
-                     : mbar_wait_cluster(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status);
-        if (!ok) break;
-        tc_fence_after();
         for (int ks = 0; ks < k_stages; ++ks, ++kcount) {
           ok = CG == 1 ? mbar_wait(bar_full + 8 * stage, phase, abort_flag, p.status)
                        : mbar_wait_cluster(bar_full + 8 * stage, phase, abort_flag, p.status);
@@ -482,16 +490,24 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
           const uint32_t sfr_lo = ((sbase + C::kOffSfR) & 0x3FFFFu) >> 4;
           const uint32_t sfb_lo = ((sbase + C::kOffSfB) & 0x3FFFFu) >> 4;
           const bool first = ks == 0;
+          // Scale-factor copies run one K step ahead of the MMAs that use them, so that the
+          // shared-memory -> tensor-memory copy of step j+1 overlaps the MMAs of step j.
+          auto copy_sf = [&](int j) {
+            tc_cp_sf<CG>(sfcol + 4 * j, ((uint64_t)kSfHi << 32) | (sfa_lo + 32 * j));
+            if (resid) tc_cp_sf<CG>(sfcol + 4 * kKSteps + 4 * j, ((uint64_t)kSfHi << 32) | (sfr_lo + 32 * j));
+            tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j, ((uint64_t)kSfHi << 32) | (sfb_lo + 32 * j));
+            tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j + 4, ((uint64_t)kSfHi << 32) | (sfb_lo + (kSfA >> 4) + 32 * j));
+          };
+          if (issuer && atoms > 0) copy_sf(0);
+          if (first) {
+            // The first scale copies of a tile do not touch the accumulator, so they are issued
+            // before waiting for the epilogue to have drained the previous tile out of it.
+            ok = CG == 1 ? mbar_wait(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status)
+                         : mbar_wait_cluster(bar_tempty, (uint32_t)(it & 1) ^ 1u, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+          }
           if (issuer) {
-            // Scale-factor copies run one K step ahead of the MMAs that use them, so that the
-            // shared-memory -> tensor-memory copy of step j+1 overlaps the MMAs of step j.
-            auto copy_sf = [&](int j) {
-              tc_cp_sf<CG>(sfcol + 4 * j, ((uint64_t)kSfHi << 32) | (sfa_lo + 32 * j));
-              if (resid) tc_cp_sf<CG>(sfcol + 4 * kKSteps + 4 * j, ((uint64_t)kSfHi << 32) | (sfr_lo + 32 * j));
-              tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j, ((uint64_t)kSfHi << 32) | (sfb_lo + 32 * j));
-              tc_cp_sf<CG>(sfcol + 8 * kKSteps + 8 * j + 4, ((uint64_t)kSfHi << 32) | (sfb_lo + (kSfA >> 4) + 32 * j));
-            };
-            if (atoms > 0) copy_sf(0);
 #pragma unroll
             for (int j = 0; j < kKSteps; ++j) {
               if (j + 1 < atoms) copy_sf(j + 1);
@@ -653,39 +669,45 @@ template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_r,
             const __grid_constant__ CUtensorMap tm_b) {
-  gemm_body<EPI, 1>(p, &tm_a, &tm_r, &tm_b);
+  gemm_body<EPI, 1>(p, &tm_a, &tm_r, &tm_b, nullptr, nullptr, nullptr);
 }
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_kernel_pair(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_r,
-                 const __grid_constant__ CUtensorMap tm_b) {
-  gemm_body<EPI, 2>(p, &tm_a, &tm_r, &tm_b);
+                 const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_sfa,
+                 const __grid_constant__ CUtensorMap tm_sfr, const __grid_constant__ CUtensorMap tm_sfb) {
+  gemm_body<EPI, 2>(p, &tm_a, &tm_r, &tm_b, &tm_sfa, &tm_sfr, &tm_sfb);
 }
 
 }  // namespace
 
-quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
-                         const CUtensorMap& tm_b, int n_sms, cudaStream_t stream) {
-  typedef void (*Fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap);
+quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const GemmMaps& m, int n_sms,
+                         cudaStream_t stream) {
   static bool attr_set[2][3] = {{false, false, false}, {false, false, false}};
-  Fn fn;
-  int smem;
-  if (cta_group == 2) {
-    fn = epi == kEpiStore ? gemm_kernel_pair<kEpiStore>
-                          : (epi == kEpiSwiGLU ? gemm_kernel_pair<kEpiSwiGLU> : gemm_kernel_pair<kEpiCombine>);
-    smem = Cfg<2>::kSmemBytes;
-  } else {
-    fn = epi == kEpiStore ? gemm_kernel<kEpiStore> : (epi == kEpiSwiGLU ? gemm_kernel<kEpiSwiGLU> : gemm_kernel<kEpiCombine>);
-    smem = Cfg<1>::kSmemBytes;
-  }
   const int g = cta_group == 2 ? 1 : 0;
-  if (!attr_set[g][epi]) {
-    QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_set[g][epi] = true;
+  if (cta_group == 2) {
+    typedef void (*Fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
+                       const CUtensorMap, const CUtensorMap);
+    Fn fn = epi == kEpiStore ? gemm_kernel_pair<kEpiStore>
+                             : (epi == kEpiSwiGLU ? gemm_kernel_pair<kEpiSwiGLU> : gemm_kernel_pair<kEpiCombine>);
+    const int smem = Cfg<2>::kSmemBytes;
+    if (!attr_set[g][epi]) {
+      QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      attr_set[g][epi] = true;
+    }
+    QUADS_CUDA_OK(launch_kernel(fn, dim3((n_sms / 2) * 2), dim3(kThreads), (size_t)smem, stream, p, m.a, m.r, m.b,
+                                m.sfa, m.sfr, m.sfb));
+  } else {
+    typedef void (*Fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap);
+    Fn fn = epi == kEpiStore ? gemm_kernel<kEpiStore> : (epi == kEpiSwiGLU ? gemm_kernel<kEpiSwiGLU> : gemm_kernel<kEpiCombine>);
+    const int smem = Cfg<1>::kSmemBytes;
+    if (!attr_set[g][epi]) {
+      QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      attr_set[g][epi] = true;
+    }
+    QUADS_CUDA_OK(launch_kernel(fn, dim3(n_sms), dim3(kThreads), (size_t)smem, stream, p, m.a, m.r, m.b));
   }
-  const int grid = cta_group == 2 ? (n_sms / 2) * 2 : n_sms;
-  QUADS_CUDA_OK(launch_kernel(fn, dim3(grid), dim3(kThreads), (size_t)smem, stream, p, tm_a, tm_r, tm_b));
   return QUADS_OK;
 }
 

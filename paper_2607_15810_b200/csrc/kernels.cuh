@@ -96,7 +96,13 @@ struct GemmParams {
   int32_t* status;       // device status word (QUADS_ERR_TIMEOUT on a failed wait)
 };
 
-quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_r,
-                         const CUtensorMap& tm_b, int n_sms, cudaStream_t stream);
+// Tensor maps of one GEMM launch: packed codes of the activation / residual / weight operands and
+// (CTA-pair variant only) their scale atoms viewed as [atoms, 128 x u32].
+struct GemmMaps {
+  CUtensorMap a, r, b, sfa, sfr, sfb;
+};
+
+quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const GemmMaps& m, int n_sms,
+                         cudaStream_t stream);
 
 }  // namespace quads

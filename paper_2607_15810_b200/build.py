@@ -32,7 +32,7 @@ def build(force=False, verbose=False):
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
         cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
                "-Xcompiler", "-fPIC", "-Xptxas", "-v" if verbose else "-O3", "-c",
-               os.path.join(CSRC, src), "-o", obj]
+               os.path.join(CSRC, src), "-o", obj] + os.environ.get("QUADS_NVCC_FLAGS", "").split()
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     for src, p in procs:

@@ -270,11 +270,6 @@ __host__ __device__ constexpr uint32_t idesc_nvf4() {
   return (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)((kBM * CG) >> 4) << 24);
 }
 
-__device__ __forceinline__ void stg256(void* addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
-                                       uint32_t f, uint32_t g, uint32_t h) {
-  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(addr), "r"(a), "r"(b), "r"(c), "r"(d),
-               "r"(e), "r"(f), "r"(g), "r"(h) : "memory");
-}
 
 struct __align__(8) BarrierBlock {
   uint64_t full[8];
@@ -313,6 +308,45 @@ __device__ __forceinline__ float warp_colsum16(const float* v, int lane) {
   float d = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 2);
   d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
   return d;
+}
+
+__device__ __forceinline__ void stg256(void* addr, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+               "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
+
+// Store a warp's 32 rows x 64 accumulator columns (thread = row) as bf16, scaled, to rows of
+// `n_out` elements starting at `dst`, rows >= rows_valid skipped.  The 32-byte chunks are first
+// transposed inside every group of 4 lanes (two butterfly exchanges), so that each store
+// instruction of the warp writes eight complete 128-byte lines instead of a 32-byte piece of 32
+// different lines.  All 32 lanes must call it.
+__device__ __forceinline__ void store_y_rows(const float* acc, float scale, uint16_t* dst, int n_out, int rows_valid,
+                                             int lane) {
+  uint32_t w[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) w[i] = f32x2_to_bf16x2(acc[2 * i] * scale, acc[2 * i + 1] * scale);
+  // chunk c = w[8c .. 8c+7]; after the exchanges chunk slot c of lane (g, j) holds chunk j of lane (g, c)
+#pragma unroll
+  for (int s = 1; s < 4; s <<= 1) {
+    const bool up = (lane & s) != 0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      if (c & s) continue;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t lo = w[8 * c + k], hi = w[8 * (c | s) + k];
+        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, up ? lo : hi, s);
+        w[8 * c + k] = up ? got : lo;
+        w[8 * (c | s) + k] = up ? hi : got;
+      }
+    }
+  }
+  const int g = lane >> 2, j = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = 4 * g + i;
+    if (r < rows_valid) stg256(dst + (size_t)r * n_out + 16 * j, w + 8 * i);
+  }
 }
 
 template <int EPI, int CG>
@@ -630,20 +664,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
         // y = W2 h~ for this dispatched row, rounded to bf16; the weighted sum over a
         // token's experts is taken afterwards in a fixed order (no atomics).
         const int n0 = nt * 256 + cq * 64;
-        if (valid && n0 < p.n_out) {
-          uint16_t* dst = p.y_pad + (size_t)prow * p.n_out + n0;
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            stg256(dst + 16 * i,
-                   f32x2_to_bf16x2(acc[16 * i] * scale, acc[16 * i + 1] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 2] * scale, acc[16 * i + 3] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 4] * scale, acc[16 * i + 5] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 6] * scale, acc[16 * i + 7] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 8] * scale, acc[16 * i + 9] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 10] * scale, acc[16 * i + 11] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 12] * scale, acc[16 * i + 13] * scale),
-                   f32x2_to_bf16x2(acc[16 * i + 14] * scale, acc[16 * i + 15] * scale));
-        }
+        if (n0 < p.n_out)
+          store_y_rows(acc, scale, p.y_pad + (size_t)(mt * kBM + q * 32) * p.n_out + n0, p.n_out, rows_of(mt) - q * 32, lane);
       } else {
         const int n0 = nt * 256 + cq * 64;
         if (valid && n0 < p.n_out) {

@@ -233,7 +233,7 @@ quads_status run_select(const float* partials, const int* n_part_ptr, int n_part
     QUADS_CUDA_OK(cudaFuncSetAttribute(rank_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
     attr = true;
   }
-  QUADS_CUDA_OK(launch_kernel(rank_select_kernel, dim3((C + 63) / 64), dim3(256), (size_t)((size_t)C * 8), st, keys, C, n_sel, mask));
+  QUADS_CUDA_OK(launch_kernel(rank_select_kernel, dim3((C + 15) / 16), dim3(256), (size_t)((size_t)C * 8), st, keys, C, n_sel, mask));
   if (sel_export) {
     QUADS_CUDA_OK(launch_kernel(sel_list_kernel, dim3(1), dim3(1024), (size_t)(0), st, mask, C, sel_export));
   }

@@ -336,8 +336,8 @@ score_reduce_kernel(const float* __restrict__ partials, const int* __restrict__ 
 // Channel selection (Eq. channel-select): rank_j = #{i : s_i > s_j, or s_i ==
 // s_j and i < j}; channel j is selected iff rank_j < n_sel (the n_sel largest,
 // ties to the lower index).  Every CTA loads all C score keys into shared
-// memory and ranks 64 channels with 4 threads each.
-// grid = ceil(C/64), 256 threads, smem = C * 8 bytes.
+// memory and ranks 16 channels with 16 threads each.
+// grid = ceil(C/16), 256 threads, smem = C * 8 bytes.
 __global__ void __launch_bounds__(256)
 rank_select_kernel(const unsigned long long* __restrict__ score_keys, int C, int n_sel, uint8_t* __restrict__ mask) {
   pdl_sync();
@@ -345,19 +345,19 @@ rank_select_kernel(const unsigned long long* __restrict__ score_keys, int C, int
   unsigned long long* sc = reinterpret_cast<unsigned long long*>(smem_raw);
   for (int i = threadIdx.x; i < C; i += blockDim.x) sc[i] = score_keys[i];
   __syncthreads();
-  const int j = blockIdx.x * 64 + (threadIdx.x >> 2);
-  const int sub = threadIdx.x & 3;
+  const int j = blockIdx.x * 16 + (threadIdx.x >> 4);
+  const int sub = threadIdx.x & 15;
   int rank = 0;
   if (j < C) {
     const unsigned long long sj = sc[j];
 #pragma unroll 8
-    for (int i = sub; i < C; i += 4) {
+    for (int i = sub; i < C; i += 16) {
       const unsigned long long si = sc[i];
       rank += (si > sj || (si == sj && i < j)) ? 1 : 0;
     }
   }
-  rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 1);
-  rank += __shfl_xor_sync(0xFFFFFFFFu, rank, 2);
+#pragma unroll
+  for (int o = 1; o < 16; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
   if (j < C && sub == 0) mask[j] = rank < n_sel ? 1 : 0;
 }
 

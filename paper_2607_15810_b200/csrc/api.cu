@@ -58,14 +58,15 @@ EncodeTiledFn encode_fn() {
 }
 
 // 2D map over packed FP4 codes viewed as bytes: [rows, row_bytes], box 128 bytes x
-// 128 rows, 128-byte swizzle, zero fill outside.
-quads_status make_codes_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes) {
+// box_rows rows, 128-byte swizzle, zero fill outside.
+quads_status make_codes_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes,
+                            uint32_t box_rows = 128) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return QUADS_ERR_CUDA;
   if (rows == 0) rows = 1;
   cuuint64_t dims[2] = {row_bytes, rows};
   cuuint64_t strides[1] = {row_bytes};
-  cuuint32_t box[2] = {(cuuint32_t)kGemmStageKBytes, 128};
+  cuuint32_t box[2] = {(cuuint32_t)kGemmStageKBytes, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -536,9 +537,13 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   trace_mark("rac_dispatch", st);
   // ---- tensor maps
+  // few rows per expert (decode-sized batches): operands swapped, weights on the M side
+  static const bool no_swap = getenv("QUADS_NO_SWAP") != nullptr;
+  const bool swapped = !dense && !no_swap && gemm_cta_group() == 1 && gemm_swapped_ok(A, E, L.m_tiles_max);
+  const uint32_t act_box = swapped ? 16 : 128;
   GemmMaps m1;
-  if ((s = make_codes_map(&m1.a, P(L.xq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&m1.r, P(L.rq_pad), pad_rows, H / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m1.a, P(L.xq_pad), pad_rows, H / 2, act_box)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m1.r, P(L.rq_pad), pad_rows, H / 2, act_box)) != QUADS_OK) return s;
   if ((s = make_codes_map(&m1.b, a->w13_q, (uint64_t)E * N1, H / 2)) != QUADS_OK) return s;
   if (gemm_cta_group() == 2) {
     const uint64_t a_atoms = (uint64_t)(pad_rows / 128) * (H / 64);
@@ -567,7 +572,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     return launch_gemm(kEpiStore, gemm_cta_group(), g, m1, di.sm_count, st);
   }
   g.n_out = I;
-  g.n_tiles_n = I / 128;
+  g.n_tiles_n = I / 128;                          // both variants: 128 features per tile (gate + up rows)
   g.half1_row_offset = I;
   g.h_gs = a->a2_gs;
   g.resid2 = a->rac_nsel_2 > 0 || a->r2q || a->r2sf;
@@ -576,7 +581,9 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.h_export = static_cast<uint16_t*>(a->h_bf16);
   const bool timing = g_timers.enabled && g_timers.created;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[0], st));
-  if ((s = launch_gemm(kEpiSwiGLU, gemm_cta_group(), g, m1, di.sm_count, st)) != QUADS_OK) return s;
+  s = swapped ? launch_gemm_swapped(kEpiSwiGLU, g, m1, di.sm_count, st)
+              : launch_gemm(kEpiSwiGLU, gemm_cta_group(), g, m1, di.sm_count, st);
+  if (s != QUADS_OK) return s;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[1], st));
 
   trace_mark("gemm1", st);
@@ -601,8 +608,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   // ---- second projection + weighted combine
   uint16_t* y_pad = reinterpret_cast<uint16_t*>(P(L.y_pad));
   GemmMaps m2;
-  if ((s = make_codes_map(&m2.a, P(L.hq_pad), pad_rows, I / 2)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&m2.r, P(L.r2q_pad), pad_rows, I / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m2.a, P(L.hq_pad), pad_rows, I / 2, act_box)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m2.r, P(L.r2q_pad), pad_rows, I / 2, act_box)) != QUADS_OK) return s;
   if ((s = make_codes_map(&m2.b, a->w2_q, (uint64_t)E * H, I / 2)) != QUADS_OK) return s;
   if (gemm_cta_group() == 2) {
     const uint64_t a_atoms = (uint64_t)(pad_rows / 128) * (I / 64);
@@ -618,11 +625,13 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g2.b_gs = a->w2_gs; g2.a_gs = a->a2_gs; g2.a_amax_bits = nullptr;
   g2.b_rows_per_expert = H;
   g2.n_out = H;
-  g2.n_tiles_n = (H + 255) / 256;
+  g2.n_tiles_n = swapped ? H / 128 : (H + 255) / 256;
   g2.half1_row_offset = 128;
   g2.y_pad = y_pad;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[2], st));
-  if ((s = launch_gemm(kEpiCombine, gemm_cta_group(), g2, m2, di.sm_count, st)) != QUADS_OK) return s;
+  s = swapped ? launch_gemm_swapped(kEpiCombine, g2, m2, di.sm_count, st)
+              : launch_gemm(kEpiCombine, gemm_cta_group(), g2, m2, di.sm_count, st);
+  if (s != QUADS_OK) return s;
   if (timing) {
     QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
     g_timers.valid = true;

@@ -102,6 +102,13 @@ struct GemmMaps {
   CUtensorMap a, r, b, sfa, sfr, sfb;
 };
 
+// Operand-swapped variant for few rows per expert (weights on the M side, tokens in chunks of 64
+// on the N side; epi = kEpiSwiGLU or kEpiCombine).  Maps: a / r = activation / residual codes with
+// boxes of 16 rows, b = weight codes with boxes of 128 rows; p.n_tiles_n counts tiles of 128
+// output features.  Usable when assignments <= 32 * experts and the slot tables fit.
+bool gemm_swapped_ok(int64_t assignments, int n_experts, int m_tiles_max);
+quads_status launch_gemm_swapped(int epi, const GemmParams& p, const GemmMaps& m, int n_sms, cudaStream_t stream);
+
 quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const GemmMaps& m, int n_sms,
                          cudaStream_t stream);
 

@@ -96,7 +96,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // ------------------------------------------------------------------ workspace
 struct MoeLayout {
-  size_t header, amax, counters13, counters2, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
+  size_t header, amax, counters13, counters2, expert_total, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
   size_t perm, pos_pad, row_token, row_weight;
   size_t partials13, scores13, keys13, keys2, sel13, mask13, xq_tok, xsf_tok, rq_tok, rsf_tok, xq_pad, xsf, rq_pad, rsf;
   size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad;
@@ -124,6 +124,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   L.amax = take(16);
   L.counters13 = take((size_t)((H + 31) / 32) * 4);
   L.counters2 = take((size_t)((I + 31) / 32 + 1) * 4);
+  L.expert_total = take((size_t)Ee * 4);           // zeroed with the header: the routing kernel adds to it
   L.ids = take((size_t)A * 4);
   L.wts = take((size_t)A * 4);
   L.chunk_counts = take((size_t)L.n_chunks * Ee * 4);
@@ -498,11 +499,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   } else {
     int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
     int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
-    QUADS_CUDA_OK(launch_kernel(route_kernel, dim3(L.n_chunks), dim3(256), (size_t)(0), rs, a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts, a->topk_ids, a->topk_w));
+    int32_t* expert_total = reinterpret_cast<int32_t*>(P(L.expert_total));
+    QUADS_CUDA_OK(launch_kernel(route_kernel, dim3(L.n_chunks), dim3(256), (size_t)(0), rs, a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts, expert_total, a->topk_ids, a->topk_w));
     trace_mark("route", st);
-    QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(1), dim3(1024), (size_t)(0), rs, E, L.n_chunks, gemm_cta_group(), chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, a->expert_offsets));
+    QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(E), dim3(256), (size_t)(0), rs, E, L.n_chunks, gemm_cta_group(), chunk_counts, expert_total, chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, a->expert_offsets));
     trace_mark("scan", st);
-    QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3((L.n_chunks + 3) / 4), dim3(128), (size_t)(0), rs, T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
+    QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3(L.n_chunks), dim3(128), (size_t)(0), rs, T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
   }
   if (side) QUADS_CUDA_OK(cudaEventRecord(side->join, side->stream));
   trace_mark("permute", st);

@@ -15,12 +15,13 @@ __device__ __forceinline__ uint32_t float_key(float v) {
 // the reduction latency).  E <= 256.  Top-k by logit, ties to the lower expert
 // id, slots in descending-logit order; weights = softmax over all experts at
 // the chosen ones, optionally renormalised.  Each CTA (kRouteTokensPerCta
-// tokens) also writes its per-expert assignment counts: chunk_counts[expert][cta].
+// tokens) also writes its per-expert assignment counts: chunk_counts[expert][cta],
+// and adds them to expert_total[expert] (zero on entry).
 constexpr int kRouteTokensPerWarp = 4;
 __global__ void __launch_bounds__(256)
 route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
              int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
-             int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
+             int32_t* __restrict__ expert_total, int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
   pdl_sync();
   __shared__ int hist[kMaxExperts];
   for (int i = threadIdx.x; i < E; i += blockDim.x) hist[i] = 0;
@@ -109,78 +110,94 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < E; i += blockDim.x) chunk_counts[(size_t)i * gridDim.x + blockIdx.x] = hist[i];
+  for (int i = threadIdx.x; i < E; i += blockDim.x) {
+    chunk_counts[(size_t)i * gridDim.x + blockIdx.x] = hist[i];
+    if (hist[i]) atomicAdd(expert_total + i, hist[i]);          // integer sums: order does not matter
+  }
 }
 
-// One CTA of 1024 threads.  A warp per expert (round robin): exclusive prefix of
-// the expert's counts over chunks and its total; then the exclusive scan over
-// experts of counts (offsets) and of 128-row tile counts (tile_prefix; every expert gets a
-// multiple of `tile_group` tiles, so that a CTA pair never straddles experts), the
-// tile -> (expert, valid rows) map, and the header.
-__global__ void __launch_bounds__(1024)
-scan_kernel(int E, int n_chunks, int tile_group, const int32_t* __restrict__ chunk_counts, int32_t* __restrict__ chunk_base,
-            int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tile_expert,
-            int32_t* __restrict__ tile_rows, int32_t* __restrict__ header, int32_t* __restrict__ offsets_out) {
+// One CTA per expert, 256 threads.  From the experts' totals: the exclusive scan over experts of
+// counts (offsets) and of 128-row tile counts (tile_prefix; every expert gets a multiple of
+// `tile_group` tiles, so that a CTA pair never straddles experts); for its own expert the
+// exclusive prefix of the counts over chunks (chunk_base) and the tile -> (expert, valid rows)
+// map; the last expert's CTA also writes the header.  E <= 256.
+__global__ void __launch_bounds__(256)
+scan_kernel(int E, int n_chunks, int tile_group, const int32_t* __restrict__ chunk_counts,
+            const int32_t* __restrict__ expert_total, int32_t* __restrict__ chunk_base, int32_t* __restrict__ offsets,
+            int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tile_expert, int32_t* __restrict__ tile_rows,
+            int32_t* __restrict__ header, int32_t* __restrict__ offsets_out) {
   pdl_sync();
-  __shared__ int cnt[kMaxExperts];
-  __shared__ int off[kMaxExperts + 1];
-  __shared__ int tpre[kMaxExperts + 1];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-  for (int e = warp; e < E; e += n_warps) {
-    int run = 0;
-    for (int c0 = 0; c0 < n_chunks; c0 += 256) {
-      int v[8];
+  __shared__ int wsum[2][8];
+  __shared__ int carry;
+  const int e = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // (1) offsets and tile prefix of this expert: block-wide sums over the experts below it
+  const int cnt = threadIdx.x < E ? expert_total[threadIdx.x] : 0;
+  const int tiles = ((cnt + 128 * tile_group - 1) / (128 * tile_group)) * tile_group;
+  int a_lo = threadIdx.x < e ? cnt : 0, t_lo = threadIdx.x < e ? tiles : 0;
+  int a_all = cnt, t_all = tiles;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {              // all loads first: one memory latency per 256 chunks
-        const int c = c0 + k * 32 + lane;
-        v[k] = c < n_chunks ? chunk_counts[(size_t)e * n_chunks + c] : 0;
-      }
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const int c = c0 + k * 32 + lane;
-        int incl = v[k];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (lane >= o) incl += n;
-        }
-        if (c < n_chunks) chunk_base[(size_t)e * n_chunks + c] = run + incl - v[k];
-        run += __shfl_sync(0xFFFFFFFFu, incl, 31);
-      }
-    }
-    if (lane == 0) cnt[e] = run;
+  for (int o = 16; o > 0; o >>= 1) {
+    a_lo += __shfl_xor_sync(0xFFFFFFFFu, a_lo, o);
+    t_lo += __shfl_xor_sync(0xFFFFFFFFu, t_lo, o);
+    a_all += __shfl_xor_sync(0xFFFFFFFFu, a_all, o);
+    t_all += __shfl_xor_sync(0xFFFFFFFFu, t_all, o);
   }
+  __shared__ int red[4][8];
+  if (lane == 0) { red[0][warp] = a_lo; red[1][warp] = t_lo; red[2][warp] = a_all; red[3][warp] = t_all; }
   __syncthreads();
+  int off_e = 0, tpre_e = 0, a_tot = 0, t_tot = 0;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) { off_e += red[0][w]; tpre_e += red[1][w]; a_tot += red[2][w]; t_tot += red[3][w]; }
+  const int my_cnt = expert_total[e];
+  const int my_tiles = ((my_cnt + 128 * tile_group - 1) / (128 * tile_group)) * tile_group;
   if (threadIdx.x == 0) {
-    int a = 0, t = 0;
-    for (int i = 0; i < E; ++i) {
-      off[i] = a; tpre[i] = t;
-      a += cnt[i];
-      t += ((cnt[i] + 128 * tile_group - 1) / (128 * tile_group)) * tile_group;
+    offsets[e] = off_e;
+    tile_prefix[e] = tpre_e;
+    if (offsets_out) offsets_out[e] = off_e;
+    if (e == E - 1) {
+      offsets[E] = a_tot;
+      tile_prefix[E] = t_tot;
+      if (offsets_out) offsets_out[E] = a_tot;
+      header[kHdrMTiles] = t_tot;
+      header[kHdrPaddedRows] = t_tot * 128;
+      header[kHdrAssignments] = a_tot;
     }
-    off[E] = a; tpre[E] = t;
-    header[kHdrMTiles] = t;
-    header[kHdrPaddedRows] = t * 128;
-    header[kHdrAssignments] = a;
   }
+  for (int m = threadIdx.x; m < my_tiles; m += blockDim.x) {
+    tile_expert[tpre_e + m] = e;
+    tile_rows[tpre_e + m] = max(0, min(128, my_cnt - m * 128));
+  }
+  // (2) exclusive prefix of this expert's counts over the chunks, 256 chunks per pass
+  if (threadIdx.x == 0) carry = 0;
   __syncthreads();
-  for (int i = threadIdx.x; i <= E; i += blockDim.x) {
-    offsets[i] = off[i];
-    tile_prefix[i] = tpre[i];
-    if (offsets_out) offsets_out[i] = off[i];
-  }
-  for (int e = warp; e < E; e += n_warps) {
-    const int n_t = tpre[e + 1] - tpre[e];
-    for (int m = lane; m < n_t; m += 32) {
-      tile_expert[tpre[e] + m] = e;
-      tile_rows[tpre[e] + m] = max(0, min(128, cnt[e] - m * 128));
+  for (int c0 = 0; c0 < n_chunks; c0 += 256) {
+    const int c = c0 + threadIdx.x;
+    const int v = c < n_chunks ? chunk_counts[(size_t)e * n_chunks + c] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += n;
     }
+    const int p = (c0 >> 8) & 1;
+    if (lane == 31) wsum[p][warp] = incl;
+    __syncthreads();
+    int before = carry;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) before += w < warp ? wsum[p][w] : 0;
+    if (c < n_chunks) chunk_base[(size_t)e * n_chunks + c] = before + incl - v;
+    __syncthreads();
+    if (threadIdx.x == 255) carry = before + incl;
+    __syncthreads();
   }
 }
 
-// One warp per routing chunk: walk the chunk's assignments in (token, slot)
-// order, 32 at a time; lanes holding the same expert rank themselves with
-// match_any, so every expert hands out consecutive rows in that order.
+// One CTA (4 warps) per routing chunk.  The chunk's assignments in (token, slot) order are split
+// into four consecutive segments, one per warp; a warp first counts its segment per expert
+// (lanes holding the same expert find each other with match_any), then every assignment's row
+// inside its expert is chunk_base + (counts of the earlier warps) + (its rank inside the warp's
+// walk), so every expert hands out consecutive rows in (token, slot) order.
 __global__ void __launch_bounds__(128)
 permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__ ids, const float* __restrict__ wts,
                const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ offsets,
@@ -189,15 +206,38 @@ permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__
   pdl_sync();
   __shared__ int run[4][kMaxExperts];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int chunk = blockIdx.x * 4 + warp;
-  if (chunk >= n_chunks) return;
-  for (int e = lane; e < E; e += 32) run[warp][e] = chunk_base[(size_t)e * n_chunks + chunk];
-  __syncwarp();
+  const int chunk = blockIdx.x;
   const int t0 = chunk * kRouteTokensPerCta;
   const int n = min(kRouteTokensPerCta, T - t0) * topk;
-  for (int i0 = 0; i0 < n; i0 += 32) {
+  const int seg = (((n + 3) / 4) + 31) & ~31;               // assignments per warp, a multiple of 32
+  const int i_begin = warp * seg, i_end = min(n, i_begin + seg);
+  for (int e = lane; e < E; e += 32) run[warp][e] = 0;
+  __syncwarp();
+  // pass 1: this warp's count per expert
+  for (int i0 = i_begin; i0 < i_end; i0 += 32) {
     const int i = i0 + lane;
-    const bool active = i < n;
+    const bool active = i < i_end;
+    const int e = active ? ids[t0 * topk + i] : (0x40000000 + lane);
+    const unsigned same = __match_any_sync(0xFFFFFFFFu, e);
+    if (active && (same & ((1u << lane) - 1u)) == 0) run[warp][e] += __popc(same);
+    __syncwarp();
+  }
+  __syncthreads();
+  // starting row of each warp inside every expert: chunk base + the earlier warps' counts
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int b = chunk_base[(size_t)e * n_chunks + chunk];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int c = run[w][e];
+      run[w][e] = b;
+      b += c;
+    }
+  }
+  __syncthreads();
+  // pass 2: hand out the rows
+  for (int i0 = i_begin; i0 < i_end; i0 += 32) {
+    const int i = i0 + lane;
+    const bool active = i < i_end;
     const int flat = t0 * topk + i;
     const int e = active ? ids[flat] : (0x40000000 + lane);
     const unsigned same = __match_any_sync(0xFFFFFFFFu, e);

@@ -196,7 +196,7 @@ inline void trace_mark(const char* name, cudaStream_t st) {
 // activation chain (amax -> quantize -> select); both are joined before the dispatch copy.
 struct SideStream {
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, mid = nullptr, join = nullptr;
   bool ok = false;
 };
 std::mutex g_side_mu;
@@ -210,6 +210,7 @@ SideStream* side_stream() {
   if (!s.ok) {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.mid, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s.ok = true;
   }
@@ -506,7 +507,6 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     trace_mark("scan", st);
     QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3(L.n_chunks), dim3(128), (size_t)(0), rs, T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
   }
-  if (side) QUADS_CUDA_OK(cudaEventRecord(side->join, side->stream));
   trace_mark("permute", st);
 
   // ---- per-tensor scale of x
@@ -522,6 +522,20 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   uint8_t* mask13 = P(L.mask13);
   QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(L.stats_ctas), dim3(H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32), (size_t)(0), st, x, T, H, a->a13_gs, amax_bits, a->a13_gs_out, L.rows_per_cta, nsel13 > 0 ? 1 : 0, reinterpret_cast<float*>(P(L.partials13)), P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), a->xq, a->xsf));
   trace_mark("rac_stats", st);
+  // The dispatched copies of Q(x) need only the dispatch order and the codes: with a side stream
+  // they are written there, next to the channel selection; the residual copies (which need the
+  // selection) follow on the main stream.
+  const int64_t scatter_chunks = (int64_t)T * (H / 32);
+  const unsigned scatter_grid = (unsigned)((scatter_chunks + 255) / 256);
+  const bool split_scatter = side != nullptr && nsel13 > 0;
+  if (side) {
+    if (split_scatter) {
+      QUADS_CUDA_OK(cudaEventRecord(side->mid, st));
+      QUADS_CUDA_OK(cudaStreamWaitEvent(side->stream, side->mid, 0));
+      QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3(scatter_grid), dim3(256), (size_t)(0), side->stream, T, H, 1, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
+    }
+    QUADS_CUDA_OK(cudaEventRecord(side->join, side->stream));
+  }
   if (nsel13 > 0) {
     s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
                    reinterpret_cast<double*>(P(L.scores13)), reinterpret_cast<unsigned int*>(P(L.counters13)),
@@ -534,8 +548,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     side_lock.unlock();
   }
   {
-    const int64_t chunks = (int64_t)T * (H / 32);
-    QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3((unsigned)((chunks + 255) / 256)), dim3(256), (size_t)(0), st, T, H, nsel13 > 0 ? 1 : 0, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
+    const int parts = split_scatter ? 2 : (nsel13 > 0 ? 3 : 1);
+    QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3(scatter_grid), dim3(256), (size_t)(0), st, T, H, parts, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
   }
   trace_mark("rac_dispatch", st);
   // ---- tensor maps

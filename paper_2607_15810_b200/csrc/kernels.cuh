@@ -29,7 +29,7 @@ __global__ void score_reduce_kernel(const float* partials, const int* n_part_ptr
                                     unsigned long long* score_keys);
 __global__ void rank_select_kernel(const unsigned long long* score_keys, int C, int n_sel, uint8_t* mask);
 __global__ void sel_list_kernel(const uint8_t* mask, int C, int32_t* sel_export);
-__global__ void rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* mask, int topk,
+__global__ void rac_scatter_kernel(int T, int H, int parts, const uint8_t* mask, int topk,
                                    const int32_t* pos_pad, const uint8_t* xq, const uint8_t* xsf, const uint8_t* rq,
                                    const uint8_t* rsf, uint8_t* xq_pad, uint8_t* xsf_tiled, uint8_t* rq_pad,
                                    uint8_t* rsf_tiled, uint8_t* rq_exp, uint8_t* rsf_exp);

@@ -404,22 +404,25 @@ __device__ __forceinline__ uint32_t nibble_mask8(const uint8_t* m) {
 }
 
 __global__ void __launch_bounds__(256)
-rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* __restrict__ mask, int topk,
+rac_scatter_kernel(int T, int H, int parts, const uint8_t* __restrict__ mask, int topk,
                    const int32_t* __restrict__ pos_pad, const uint8_t* __restrict__ xq,
                    const uint8_t* __restrict__ xsf, const uint8_t* __restrict__ rq, const uint8_t* __restrict__ rsf,
                    uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled, uint8_t* __restrict__ rq_pad,
                    uint8_t* __restrict__ rsf_tiled, uint8_t* __restrict__ rq_exp, uint8_t* __restrict__ rsf_exp) {
   pdl_sync();
   const int per_row = H >> 5;                         // 16-byte chunks of codes per row
-  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= (int64_t)T * per_row) return;
+  const int64_t n_chunks = (int64_t)T * per_row;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_chunks; g += (int64_t)gridDim.x * blockDim.x) {
   const int t = (int)(g / per_row), c = (int)(g - (int64_t)t * per_row);
   const size_t co = (size_t)t * (H >> 1) + c * 16;
-  const uint4 xv = __ldg(reinterpret_cast<const uint4*>(xq + co));
-  uint4 rv = make_uint4(0, 0, 0, 0);
+  const bool do_x = (parts & 1) != 0, with_residual = (parts & 2) != 0;
+  uint4 xv = make_uint4(0, 0, 0, 0), rv = make_uint4(0, 0, 0, 0);
   const bool sf_owner = (c & 1) == 0;                 // even chunks also move 4 scale bytes (64 channels)
   uint32_t xs = 0, rs = 0;
-  if (sf_owner) xs = __ldg(reinterpret_cast<const uint32_t*>(xsf + (size_t)t * (H >> 4) + c * 2));
+  if (do_x) {
+    xv = __ldg(reinterpret_cast<const uint4*>(xq + co));
+    if (sf_owner) xs = __ldg(reinterpret_cast<const uint32_t*>(xsf + (size_t)t * (H >> 4) + c * 2));
+  }
   if (with_residual) {
     rv = __ldg(reinterpret_cast<const uint4*>(rq + co));
     const uint8_t* m = mask + c * 32;
@@ -439,14 +442,15 @@ rac_scatter_kernel(int T, int H, int with_residual, const uint8_t* __restrict__ 
     for (int j = 0; j < 8; ++j) {
       if (p[j] < 0) continue;
       const size_t po = (size_t)p[j] * (H >> 1) + c * 16;
-      __stcs(reinterpret_cast<uint4*>(xq_pad + po), xv);
+      if (do_x) __stcs(reinterpret_cast<uint4*>(xq_pad + po), xv);
       if (with_residual) __stcs(reinterpret_cast<uint4*>(rq_pad + po), rv);
       if (sf_owner) {
         const size_t so = sf_tiled_offset(p[j], c * 2, kt_count);
-        *reinterpret_cast<uint32_t*>(xsf_tiled + so) = xs;
+        if (do_x) *reinterpret_cast<uint32_t*>(xsf_tiled + so) = xs;
         if (with_residual) *reinterpret_cast<uint32_t*>(rsf_tiled + so) = rs;
       }
     }
+  }
   }
 }
 

@@ -391,6 +391,31 @@ def run_ours(args):
         aux["fake_quant_frac_of_hbm"] = aux["fake_quant_gbs"] / peaks["hbm_gbs"]
         aux["hbm_peak_gbs"] = peaks["hbm_gbs"]
         del w, outs
+        # decode-sized batch on the same layer (the prefill and decode workloads share their weights):
+        # weights cold (L2 flushed between iterations); roofline = streaming the 340 MB of weights once
+        if args.workload == "prefill":
+            dsh = synth.MOE_SHAPES["decode"]
+            dn13, dn2 = nsel_of(dsh, args.variant)
+            dx, _ = synth.activations(dsh)
+            dlg = synth.router_logits(dsh)
+            dx, dlg = dx.to(dev), dlg.to(dev)
+            da2 = torch.tensor([synth.H_GLOBAL_SCALE[dsh.name]], dtype=torch.float32, device=dev)
+            dws = torch.empty(B.moe_workspace_bytes(dsh.T, dsh.H, dsh.I, dsh.E, dsh.topk), dtype=torch.uint8, device=dev)
+            dout = torch.empty(dsh.T, dsh.H, dtype=torch.bfloat16, device=dev)
+
+            def dstep():
+                B.moe_w4a4_rac(dx, dlg, gw13, gw2, dsh.topk, dn13, dn2, da2, workspace=dws, out=dout)
+            for _ in range(5):
+                flush.fill_(1)
+                dstep()
+            td = timed(dstep, 50)
+            dms = sum(td) / len(td)
+            wbytes = sum(t.numel() * t.element_size() for g in (gw13, gw2) for t in g.values())
+            aux["decode_ms_per_step"] = dms
+            aux["decode_tokens_per_s"] = dsh.T / (dms * 1e-3)
+            aux["decode_weight_stream_gbs"] = wbytes / (dms * 1e-3) / 1e9
+            aux["decode_frac_of_hbm"] = aux["decode_weight_stream_gbs"] / peaks["hbm_gbs"]
+            aux["decode_note"] = "T=%d on the same layer, cold weights (%.0f MB streamed per step)" % (dsh.T, wbytes / 1e6)
         line["aux"] = aux
 
     if world == 1 and not args.no_cpu_baseline:

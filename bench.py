@@ -416,6 +416,16 @@ def run_ours(args):
             aux["decode_weight_stream_gbs"] = wbytes / (dms * 1e-3) / 1e9
             aux["decode_frac_of_hbm"] = aux["decode_weight_stream_gbs"] / peaks["hbm_gbs"]
             aux["decode_note"] = "T=%d on the same layer, cold weights (%.0f MB streamed per step)" % (dsh.T, wbytes / 1e6)
+            # the same call replayed from a CUDA graph (what a decode loop does)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                dstep()
+            for _ in range(3):
+                flush.fill_(1)
+                graph.replay()
+            tg = timed(graph.replay, 50)
+            aux["decode_graph_ms_per_step"] = sum(tg) / len(tg)
+            aux["decode_graph_tokens_per_s"] = dsh.T / (aux["decode_graph_ms_per_step"] * 1e-3)
         line["aux"] = aux
 
     if world == 1 and not args.no_cpu_baseline:

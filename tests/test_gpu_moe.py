@@ -233,3 +233,47 @@ def test_cta_pair_gemm_variant_in_a_subprocess():
                         "gpu", "-k", "dense_config_all_ratios or dense_ragged or small_layers or edge_shapes"],
                        cwd=root, env=env, capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-3000:]
+
+
+def test_moe_call_is_capturable_in_a_cuda_graph(B):
+    """The layer call allocates nothing and never synchronises, so (after one
+    eager call has set the kernels' attributes) it can be captured into a CUDA
+    graph; replays on new inputs reproduce the eager results bit for bit."""
+    sh = synth.MOE_SHAPES["tiny"]
+    w13 = synth.expert_weights(sh, "w13")
+    w2 = synth.expert_weights(sh, "w2")
+    gw13 = B.fake_quant_weights(w13.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    gw2 = B.fake_quant_weights(w2.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    x0, _ = synth.activations(sh)
+    lg0 = synth.router_logits(sh)
+    a2 = torch.tensor([0.25], device="cuda")
+    nsel13, nsel2 = sh.H // 2, sh.I // 2
+    ws = torch.empty(B.moe_workspace_bytes(sh.T, sh.H, sh.I, sh.E, sh.topk), dtype=torch.uint8, device="cuda")
+    x_s, lg_s = x0.cuda().clone(), lg0.cuda().clone()
+    out_s = torch.empty(sh.T, sh.H, dtype=torch.bfloat16, device="cuda")
+
+    def call(x, lg, out):
+        B.moe_w4a4_rac(x, lg, gw13, gw2, sh.topk, nsel13, nsel2, a2, workspace=ws, out=out)
+
+    inputs = []
+    g = torch.Generator().manual_seed(77)
+    for i in range(3):
+        x = (x0.float() * (1.0 + 0.1 * i) + 0.01 * torch.randn(x0.shape, generator=g)).to(torch.bfloat16)
+        lg = lg0 + 0.5 * torch.randn(lg0.shape, generator=g)
+        inputs.append((x.cuda(), lg.cuda()))
+    eager = []
+    for x, lg in inputs:
+        o = torch.empty_like(out_s)
+        call(x, lg, o)
+        torch.cuda.synchronize()
+        eager.append(o.clone())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call(x_s, lg_s, out_s)
+    for (x, lg), want in zip(inputs, eager):
+        x_s.copy_(x)
+        lg_s.copy_(lg)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert B.moe_async_status(ws) == 0
+        assert torch.equal(out_s, want)

@@ -1,6 +1,7 @@
 // C ABI entry points: argument checks, workspace carving, TMA descriptors and
 // the launch sequence of each public call.
 #include <cstdlib>
+#include <atomic>
 #include <mutex>
 
 #include "kernels.cuh"
@@ -231,11 +232,7 @@ quads_status run_select(const float* partials, const int* n_part_ptr, int n_part
                         int n_sel, double* slice_sums, unsigned int* counters, unsigned long long* keys,
                         uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
   QUADS_CUDA_OK(launch_kernel(score_reduce_kernel, dim3((C + 31) / 32, kScoreSlices), dim3(256), (size_t)(0), st, partials, n_part_ptr, n_part_mul, n_part_fixed, C, slice_sums, counters, keys));
-  static bool attr = false;
-  if (!attr) {
-    QUADS_CUDA_OK(cudaFuncSetAttribute(rank_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-    attr = true;
-  }
+  QUADS_CUDA_OK(set_max_dynamic_smem<rank_select_kernel>(128 * 1024));
   QUADS_CUDA_OK(launch_kernel(rank_select_kernel, dim3((C + 15) / 16), dim3(256), (size_t)((size_t)C * 8), st, keys, C, n_sel, mask));
   if (sel_export) {
     QUADS_CUDA_OK(launch_kernel(sel_list_kernel, dim3(1), dim3(1024), (size_t)(0), st, mask, C, sel_export));
@@ -302,11 +299,13 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   int tiled = sf_layout == QUADS_SF_TILED;
   int64_t sf_stride = tiled ? (int64_t)quads_sf_tiled_bytes(rows, K) : rows * (K / 16);
   const int64_t nblk = rows * (K / 16);
-  static int blocks_per_sm = 0;
+  static std::atomic<int> blocks_per_sm_cache{0};   // same kernel and block size on every sm_100 device
+  int blocks_per_sm = blocks_per_sm_cache.load();
   if (blocks_per_sm == 0) {
     int b = 0;
     QUADS_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, fused_quantize_kernel, 256, 0));
     blocks_per_sm = b < 1 ? 1 : (b > 8 ? 8 : b);
+    blocks_per_sm_cache.store(blocks_per_sm);
   }
   int max_groups = 4;
   int n_groups = n_tensors < max_groups ? (int)n_tensors : max_groups;

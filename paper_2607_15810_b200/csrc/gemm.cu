@@ -515,33 +515,31 @@ gemm_kernel_pair(const GemmParams p, const __grid_constant__ CUtensorMap tm_a, c
 
 }  // namespace
 
+template <int EPI>
+quads_status launch_one(const GemmParams& p, const GemmMaps& m, int n_sms, cudaStream_t stream) {
+  QUADS_CUDA_OK(set_max_dynamic_smem<gemm_kernel<EPI>>(Cfg<1>::kSmemBytes));
+  QUADS_CUDA_OK(launch_kernel(gemm_kernel<EPI>, dim3(n_sms), dim3(kThreads), (size_t)Cfg<1>::kSmemBytes, stream, p, m.a,
+                              m.r, m.b));
+  return QUADS_OK;
+}
+template <int EPI>
+quads_status launch_pair(const GemmParams& p, const GemmMaps& m, int n_sms, cudaStream_t stream) {
+  QUADS_CUDA_OK(set_max_dynamic_smem<gemm_kernel_pair<EPI>>(Cfg<2>::kSmemBytes));
+  QUADS_CUDA_OK(launch_kernel(gemm_kernel_pair<EPI>, dim3((n_sms / 2) * 2), dim3(kThreads), (size_t)Cfg<2>::kSmemBytes,
+                              stream, p, m.a, m.r, m.b, m.sfa, m.sfr, m.sfb));
+  return QUADS_OK;
+}
+
 quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const GemmMaps& m, int n_sms,
                          cudaStream_t stream) {
-  static bool attr_set[2][3] = {{false, false, false}, {false, false, false}};
-  const int g = cta_group == 2 ? 1 : 0;
   if (cta_group == 2) {
-    typedef void (*Fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
-                       const CUtensorMap, const CUtensorMap);
-    Fn fn = epi == kEpiStore ? gemm_kernel_pair<kEpiStore>
-                             : (epi == kEpiSwiGLU ? gemm_kernel_pair<kEpiSwiGLU> : gemm_kernel_pair<kEpiCombine>);
-    const int smem = Cfg<2>::kSmemBytes;
-    if (!attr_set[g][epi]) {
-      QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-      attr_set[g][epi] = true;
-    }
-    QUADS_CUDA_OK(launch_kernel(fn, dim3((n_sms / 2) * 2), dim3(kThreads), (size_t)smem, stream, p, m.a, m.r, m.b,
-                                m.sfa, m.sfr, m.sfb));
-  } else {
-    typedef void (*Fn)(const GemmParams, const CUtensorMap, const CUtensorMap, const CUtensorMap);
-    Fn fn = epi == kEpiStore ? gemm_kernel<kEpiStore> : (epi == kEpiSwiGLU ? gemm_kernel<kEpiSwiGLU> : gemm_kernel<kEpiCombine>);
-    const int smem = Cfg<1>::kSmemBytes;
-    if (!attr_set[g][epi]) {
-      QUADS_CUDA_OK(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-      attr_set[g][epi] = true;
-    }
-    QUADS_CUDA_OK(launch_kernel(fn, dim3(n_sms), dim3(kThreads), (size_t)smem, stream, p, m.a, m.r, m.b));
+    return epi == kEpiStore ? launch_pair<kEpiStore>(p, m, n_sms, stream)
+                            : (epi == kEpiSwiGLU ? launch_pair<kEpiSwiGLU>(p, m, n_sms, stream)
+                                                 : launch_pair<kEpiCombine>(p, m, n_sms, stream));
   }
-  return QUADS_OK;
+  return epi == kEpiStore ? launch_one<kEpiStore>(p, m, n_sms, stream)
+                          : (epi == kEpiSwiGLU ? launch_one<kEpiSwiGLU>(p, m, n_sms, stream)
+                                               : launch_one<kEpiCombine>(p, m, n_sms, stream));
 }
 
 }  // namespace quads

@@ -412,21 +412,12 @@ bool gemm_swapped_ok(int64_t assignments, int n_experts, int m_tiles_max) {
 }
 
 quads_status launch_gemm_swapped(int epi, const GemmParams& p, const GemmMaps& m, int n_sms, cudaStream_t stream) {
-  static bool attr_set[2] = {false, false};
   if (epi == kEpiSwiGLU) {
-    if (!attr_set[0]) {
-      QUADS_CUDA_OK(cudaFuncSetAttribute(gemm_swapped_kernel<kEpiSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SCfg<kEpiSwiGLU>::kSmemBytes));
-      attr_set[0] = true;
-    }
+    QUADS_CUDA_OK(set_max_dynamic_smem<gemm_swapped_kernel<kEpiSwiGLU>>(SCfg<kEpiSwiGLU>::kSmemBytes));
     QUADS_CUDA_OK(launch_kernel(gemm_swapped_kernel<kEpiSwiGLU>, dim3(n_sms), dim3(kThreads),
                                 (size_t)SCfg<kEpiSwiGLU>::kSmemBytes, stream, p, m.a, m.r, m.b));
   } else {
-    if (!attr_set[1]) {
-      QUADS_CUDA_OK(cudaFuncSetAttribute(gemm_swapped_kernel<kEpiCombine>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SCfg<kEpiCombine>::kSmemBytes));
-      attr_set[1] = true;
-    }
+    QUADS_CUDA_OK(set_max_dynamic_smem<gemm_swapped_kernel<kEpiCombine>>(SCfg<kEpiCombine>::kSmemBytes));
     QUADS_CUDA_OK(launch_kernel(gemm_swapped_kernel<kEpiCombine>, dim3(n_sms), dim3(kThreads),
                                 (size_t)SCfg<kEpiCombine>::kSmemBytes, stream, p, m.a, m.r, m.b));
   }

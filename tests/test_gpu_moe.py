@@ -114,6 +114,11 @@ EDGE_SHAPES = [
     synth.MoEShape("one_expert", 33, 300, 128, 1, 1, 256, 0.05, 1, 3.0, 10.0),
     # K tails: H and I that are not multiples of the 256-element pipeline stage
     synth.MoEShape("k_tail", 34, 70, 384, 4, 2, 128, 0.05, 2, 3.0, 10.0),
+    # more than 256 routing chunks (second pass of the per-expert chunk scan), dozens of tiles per expert
+    synth.MoEShape("many_chunks", 35, 8300, 128, 4, 2, 128, 0.05, 1, 3.0, 10.0),
+    # few rows per expert on average (operand-swapped GEMMs) but one hot expert whose slot uses
+    # both 64-row halves and a second slot
+    synth.MoEShape("hot_expert_few_rows", 36, 200, 256, 16, 2, 128, 0.05, 2, 3.0, 10.0, 1, 0.45),
 ]
 
 

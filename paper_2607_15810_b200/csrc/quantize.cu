@@ -455,13 +455,30 @@ rac_scatter_kernel(int T, int H, int parts, const uint8_t* __restrict__ mask, in
 }
 
 // Clear (in place) the codes of unselected channels of a padded [rows, C/2]
-// code matrix; one thread per 16 bytes (32 channels).
+// code matrix; one thread per 16 bytes (32 channels).  A thread keeps its column
+// chunk (its four nibble-mask words are formed once) and walks down the rows.
 __global__ void __launch_bounds__(256)
 mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_ptr, int C,
                   const uint8_t* __restrict__ mask) {
   pdl_sync();
   const int per_row = C >> 5;
-  const int64_t n = (int64_t)(*n_rows_ptr) * per_row;
+  const int n_rows = *n_rows_ptr;
+  if (per_row <= 256) {
+    const int rows_per_pass = 256 / per_row;
+    const int c = threadIdx.x % per_row, rl = threadIdx.x / per_row;
+    if (rl >= rows_per_pass) return;
+    const uint8_t* m = mask + c * 32;
+    const uint32_t m0 = nibble_mask8(m), m1 = nibble_mask8(m + 8), m2 = nibble_mask8(m + 16), m3 = nibble_mask8(m + 24);
+    if ((m0 & m1 & m2 & m3) == 0xFFFFFFFFu) return;          // every channel of this chunk is selected
+    for (int r = blockIdx.x * rows_per_pass + rl; r < n_rows; r += gridDim.x * rows_per_pass) {
+      uint4* p = reinterpret_cast<uint4*>(codes + (size_t)r * (C >> 1)) + c;
+      uint4 v = *p;
+      v.x &= m0; v.y &= m1; v.z &= m2; v.w &= m3;
+      *p = v;
+    }
+    return;
+  }
+  const int64_t n = (int64_t)n_rows * per_row;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const int c = (int)(i % per_row);
     uint4* p = reinterpret_cast<uint4*>(codes) + i;

@@ -509,7 +509,17 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   trace_mark("permute", st);
 
   // ---- per-tensor scale of x
-  if (!a->a13_gs) {
+  // ---- per-tensor scale of x: folded into the quantization kernel (cooperative launch, grid
+  // barrier) when all of its CTAs fit on the GPU at once; else a kernel of its own
+  const int rq_block = H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32;
+  static const bool no_fused_amax = getenv("QUADS_NO_FUSED_AMAX") != nullptr;
+  bool fused_amax = false;
+  if (!a->a13_gs && !no_fused_amax && !g_trace.enabled) {
+    int per_sm = 0;
+    QUADS_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rac_quant_kernel, rq_block, 0));
+    fused_amax = (int64_t)per_sm * di.sm_count >= L.stats_ctas;
+  }
+  if (!a->a13_gs && !fused_amax) {
     const int64_t chunks = (int64_t)T * (H / 8);
     int gx = (int)((chunks + 2047) / 2048);
     if (gx > di.sm_count * 8) gx = di.sm_count * 8;
@@ -519,7 +529,28 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   // ---- site 13: quantize (+ residual + statistics), selection, dispatch scatter
   const int nsel13 = a->rac_nsel_13;
   uint8_t* mask13 = P(L.mask13);
-  QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(L.stats_ctas), dim3(H / 16 > 256 ? 256 : (H / 16 + 31) / 32 * 32), (size_t)(0), st, x, T, H, a->a13_gs, amax_bits, a->a13_gs_out, L.rows_per_cta, nsel13 > 0 ? 1 : 0, reinterpret_cast<float*>(P(L.partials13)), P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), a->xq, a->xsf));
+  {
+    const uint16_t* xp = x;
+    int Tt = T, Hh = H, rows_per_cta = L.rows_per_cta, with_res = nsel13 > 0 ? 1 : 0;
+    const float* gs13 = a->a13_gs;
+    unsigned int* arrivals = fused_amax ? reinterpret_cast<unsigned int*>(header + kHdrArrivals) : nullptr;
+    int32_t* status_word = header + kHdrStatus;
+    float* gs_store = a->a13_gs_out;
+    float* partials = reinterpret_cast<float*>(P(L.partials13));
+    uint8_t *xq_tok = P(L.xq_tok), *xsf_tok = P(L.xsf_tok), *rq_tok = P(L.rq_tok), *rsf_tok = P(L.rsf_tok);
+    uint8_t *xq_exp = a->xq, *xsf_exp = a->xsf;
+    if (fused_amax) {
+      void* args[] = {&xp, &Tt, &Hh, &gs13, &amax_bits, &arrivals, &status_word, &gs_store, &rows_per_cta, &with_res,
+                      &partials, &xq_tok, &xsf_tok, &rq_tok, &rsf_tok, &xq_exp, &xsf_exp};
+      QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(rac_quant_kernel), dim3(L.stats_ctas),
+                                                dim3(rq_block), args, 0, st));
+      note_launch();
+    } else {
+      QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(L.stats_ctas), dim3(rq_block), (size_t)(0), st, xp, Tt, Hh, gs13,
+                                  amax_bits, arrivals, status_word, gs_store, rows_per_cta, with_res, partials, xq_tok,
+                                  xsf_tok, rq_tok, rsf_tok, xq_exp, xsf_exp));
+    }
+  }
   trace_mark("rac_stats", st);
   // The dispatched copies of Q(x) need only the dispatch order and the codes: with a side stream
   // they are written there, next to the channel selection; the residual copies (which need the

@@ -11,7 +11,7 @@ constexpr int kMaxTopk = 16;
 constexpr int kMaxExperts = 256;
 
 // header words written by the scan (device side sizes of the dispatch)
-enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, kHdrWords = 8 };
+enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, kHdrArrivals = 4, kHdrWords = 8 };
 
 // ---- quantize.cu
 __global__ void amax_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
@@ -20,7 +20,8 @@ __global__ void fused_quantize_kernel(const uint16_t* x, int64_t rows, int64_t K
                                       int n_tensors, const float* gs_in, uint32_t* amax_bits, uint32_t* counters,
                                       uint8_t* q, uint8_t* sf, uint16_t* fq, float* gs_out, int sf_tiled,
                                       int64_t sf_tensor_stride, int n_groups);
-__global__ void rac_quant_kernel(const uint16_t* x, int T, int H, const float* gs_in, const uint32_t* amax_bits,
+__global__ void rac_quant_kernel(const uint16_t* x, int T, int H, const float* gs_in, uint32_t* amax_bits,
+                                 unsigned int* grid_arrivals, int32_t* status,
                                  float* gs_store, int rows_per_cta, int with_residual, float* partials, uint8_t* xq,
                                  uint8_t* xsf, uint8_t* rq, uint8_t* rsf, uint8_t* xq_exp, uint8_t* xsf_exp);
 constexpr int kScoreSlices = 16;

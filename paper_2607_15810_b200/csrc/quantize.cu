@@ -236,12 +236,55 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __restrict__ gs_in,
-                 const uint32_t* __restrict__ amax_bits, float* __restrict__ gs_store, int rows_per_cta,
+                 uint32_t* __restrict__ amax_bits, unsigned int* __restrict__ grid_arrivals, int32_t* __restrict__ status,
+                 float* __restrict__ gs_store, int rows_per_cta,
                  int with_residual, float* __restrict__ partials, uint8_t* __restrict__ xq,
                  uint8_t* __restrict__ xsf, uint8_t* __restrict__ rq, uint8_t* __restrict__ rsf,
                  uint8_t* __restrict__ xq_exp, uint8_t* __restrict__ xsf_exp) {
   pdl_sync();
-  const float gs = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
+  const int k16 = H >> 4;
+  const int r0 = blockIdx.x * rows_per_cta;
+  const int r1 = min(T, r0 + rows_per_cta);
+  __shared__ float gs_sh;
+  if (grid_arrivals) {
+    // Cooperative launch with no per-tensor scale given: first the tensor's amax over this
+    // CTA's rows (the same rows it quantizes below, so the second read hits L1 / L2), then a
+    // bounded wait until every CTA has contributed.
+    __shared__ uint32_t wmax[8];
+    uint32_t m = 0;
+    for (int kb = threadIdx.x; kb < k16; kb += blockDim.x)
+      for (int r = r0; r < r1; ++r) {
+        uint4 v0, v1;
+        ldg256(x + (size_t)r * H + kb * 16, v0, v1);
+        m = __vmaxu2(m, __vmaxu2(absmax8(v0), absmax8(v1)));
+      }
+    uint32_t smx = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) smx = max(smx, __shfl_xor_sync(0xFFFFFFFFu, smx, o));
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = smx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t tm = 0;
+      for (int i = 0; i < (int)((blockDim.x + 31) >> 5); ++i) tm = max(tm, wmax[i]);
+      if (tm) atomicMax(amax_bits, tm << 16);
+      __threadfence();
+      atomicAdd(grid_arrivals, 1u);
+      const long long t0 = clock64();
+      unsigned int seen;
+      for (;;) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(grid_arrivals) : "memory");
+        if (seen >= gridDim.x) break;
+        __nanosleep(200);
+        if (clock64() - t0 > 4000000000ll) { atomicExch(status, (int32_t)QUADS_ERR_TIMEOUT); break; }
+      }
+      gs_sh = gs_from_amax_bits(atomicAdd(amax_bits, 0u));
+    }
+    __syncthreads();
+  } else if (threadIdx.x == 0) {
+    gs_sh = gs_in ? gs_in[0] : gs_from_amax_bits(amax_bits[0]);
+  }
+  __syncthreads();
+  const float gs = gs_sh;
   if (gs_store && blockIdx.x == 0 && threadIdx.x == 0) gs_store[0] = gs;
   __shared__ float inv_lut[128];
   for (int i = threadIdx.x; i < 128; i += blockDim.x) inv_lut[i] = quant_inv_entry(i, gs);
@@ -249,9 +292,6 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
   QuantCtx qc;
   quant_ctx_scalars(qc, gs);
   qc.inv_lut = inv_lut;
-  const int k16 = H >> 4;
-  const int r0 = blockIdx.x * rows_per_cta;
-  const int r1 = min(T, r0 + rows_per_cta);
   for (int kb = threadIdx.x; kb < k16; kb += blockDim.x) {
     float acc[16];
 #pragma unroll

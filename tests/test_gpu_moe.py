@@ -47,7 +47,10 @@ def test_dense_config_all_ratios(B, nsel):
 
 
 @pytest.mark.parametrize("T,K,N,nsel,seed", [(1, 128, 128, 8, 1), (200, 640, 384, 64, 5), (300, 2048, 512, 1024, 6),
-                                             (129, 384, 128, 96, 7)])
+                                             (129, 384, 128, 96, 7),
+                                             # the widest layer the library takes (K = 16384: 64 pipeline stages
+                                             # per tile, 128 KB of score keys in the selection kernel)
+                                             (64, 16384, 128, 4096, 8)])
 def test_dense_ragged_shapes(B, T, K, N, nsel, seed):
     x, w = synth.dense_inputs(seed, T=T, K=K, N=N)
     _dense_case(B, x, w, nsel)

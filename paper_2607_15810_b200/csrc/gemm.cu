@@ -13,9 +13,9 @@
 //
 // Two variants share the code: CG = 1 (one CTA per tile of 128 x 256) and CG = 2
 // (a cluster of two CTAs computes a 256 x 256 tile with `cta_group::2` MMAs:
-// each CTA holds its own 128 rows of A^ / R^ and HALF of the weight tile, so the
-// bytes every SM must pull from L2 per flop drop by about a quarter -- the
-// single-CTA kernel is bound by exactly that ingest, not by the tensor pipe).
+// each CTA holds its own 128 rows of A^ / R^ and HALF of the weight tile, and one
+// thread issues the MMAs and scale copies of both SMs; per 128-row tile it is about a
+// tenth faster, but every expert's rows must then be padded to a multiple of 256).
 // No TMA multicast is used: every CTA loads what it needs itself.
 //
 // One persistent CTA per SM, 18 warps:

@@ -401,6 +401,34 @@ def run_ours(args):
         aux["fake_quant_frac_of_hbm"] = aux["fake_quant_gbs"] / peaks["hbm_gbs"]
         aux["hbm_peak_gbs"] = peaks["hbm_gbs"]
         del w, outs
+        # one whole layer of the AQAT + weight-sync workload: 128 experts x (W13 [3072, 4096] + W2 [4096, 1536]),
+        # 2.416 G elements = 4.83 GB in, 6.19 GB out; the 48-layer job is this 48 times over one reused buffer
+        torch.cuda.empty_cache()
+        n_e = 128
+        w13l = torch.empty(n_e, 3072, 4096, dtype=torch.bfloat16, device=dev)
+        w2l = torch.empty(n_e, 4096, 1536, dtype=torch.bfloat16, device=dev)
+        for wl in (w13l, w2l):
+            for e0 in range(0, n_e, 16):
+                wl[e0:e0 + 16].copy_((torch.randn(16, *wl.shape[1:], device=dev) * 0.015).to(torch.bfloat16))
+        outs13 = (torch.empty_like(w13l), torch.empty(n_e, 3072, 2048, dtype=torch.uint8, device=dev),
+                  torch.empty(n_e, 3072, 256, dtype=torch.uint8, device=dev), torch.empty(n_e, dtype=torch.float32, device=dev))
+        outs2 = (torch.empty_like(w2l), torch.empty(n_e, 4096, 768, dtype=torch.uint8, device=dev),
+                 torch.empty(n_e, 4096, 96, dtype=torch.uint8, device=dev), torch.empty(n_e, dtype=torch.float32, device=dev))
+        lws = torch.empty(B.lib.quads_fake_quant_workspace_bytes(n_e), dtype=torch.uint8, device=dev)
+
+        def layer_step():
+            B.fake_quant_weights(w13l, out=outs13, workspace=lws)
+            B.fake_quant_weights(w2l, out=outs2, workspace=lws)
+        layer_step()
+        tl = timed(layer_step, 3, with_flush=False)
+        lms = sum(tl) / len(tl)
+        n_el = w13l.numel() + w2l.numel()
+        aux["aqat_layer_ms"] = lms
+        aux["aqat_layer_gbs"] = n_el * 4.5625 / (lms * 1e-3) / 1e9
+        aux["aqat_layer_frac_of_hbm"] = aux["aqat_layer_gbs"] / peaks["hbm_gbs"]
+        aux["aqat_48_layers_s_extrapolated"] = 48 * lms * 1e-3
+        del w13l, w2l, outs13, outs2
+        torch.cuda.empty_cache()
         # decode-sized batch on the same layer (the prefill and decode workloads share their weights):
         # weights cold (L2 flushed between iterations); roofline = streaming the 340 MB of weights once
         if args.workload == "prefill":

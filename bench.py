@@ -286,6 +286,49 @@ def run_ours(args):
     e2e_times = timed(e2e_step, args.steps)
     barrier()
     e2e_ms = max_over_ranks(sum(e2e_times) / len(e2e_times))
+
+    # the same end-to-end work pipelined across steps, as a serving loop runs it: every step still
+    # copies its own inputs from pinned host memory and its own result back, but on copy streams
+    # of their own (two device buffers each way), so a step's transfers overlap its neighbours' compute
+    s_in, s_out, s_cmp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+    xin = [torch.empty_like(x_d) for _ in range(2)]
+    lgin = [torch.empty_like(lg_d) for _ in range(2)]
+    outb = [torch.empty_like(out_d) for _ in range(2)]
+
+    def pipelined(k):
+        ev_in = [torch.cuda.Event() for _ in range(k)]
+        ev_cmp = [torch.cuda.Event() for _ in range(k)]
+        ev_out = [torch.cuda.Event() for _ in range(k)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s_in.wait_stream(s_cmp)
+        s_out.wait_stream(s_cmp)
+        t0.record(s_in)
+        for i in range(k):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_cmp[i - 2])          # the input buffer has been consumed
+                xin[b].copy_(x_h, non_blocking=True)
+                lgin[b].copy_(lg_h, non_blocking=True)
+                ev_in[i].record(s_in)
+            s_cmp.wait_event(ev_in[i])
+            if i >= 2:
+                s_cmp.wait_event(ev_out[i - 2])             # the output buffer has been read back
+            flush.fill_(1)
+            B.moe_w4a4_rac(xin[b], lgin[b], gw13, gw2, topk, n13, n2, a2, workspace=ws, out=outb[b])
+            ev_cmp[i].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_cmp[i])
+                out_h.copy_(outb[b], non_blocking=True)
+                ev_out[i].record(s_out)
+        t1.record(s_out)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / k
+
+    pipelined(4)
+    barrier()
+    e2e_pipe_ms = max_over_ranks(pipelined(args.steps))
+    barrier()
     clocks = sampler.stop() if sampler else None
 
     # per-kernel time of the two grouped GEMMs (events recorded by the library on the launch stream)
@@ -336,8 +379,11 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "fp4 (e2m1 x e2m1, ue4m3 block scales, fp32 accumulate)",
             "data": "synthetic", "config": workload_config(shape, args.variant),
             "clocks": clocks, "wall_s_timed_region": wall,
-            "e2e": {"value": D.whole_job_rate(world, T, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": x_h.numel() * 2 + lg_h.numel() * 4, "d2h_bytes_per_step": out_h.numel() * 2},
+            "e2e": {"value": D.whole_job_rate(world, T, e2e_pipe_ms), "unit": UNIT, "ms_per_step": e2e_pipe_ms,
+                    "h2d_bytes_per_step": x_h.numel() * 2 + lg_h.numel() * 4, "d2h_bytes_per_step": out_h.numel() * 2,
+                    "how": "every step copies its inputs from pinned host memory and its result back; copies run on "
+                           "their own streams with two device buffers each way, so they overlap neighbouring steps",
+                    "serial_value": D.whole_job_rate(world, T, e2e_ms), "serial_ms_per_step": e2e_ms},
             "gpu_launches": launches_per_step * args.steps,
             "tflops": {"model": f_model / (ms * 1e-3) / 1e12, "algorithmic": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12,
                        "frac_of_fp4_peak": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12 / fp4_peak},

@@ -475,6 +475,24 @@ def run_ours(args):
         aux["aqat_48_layers_s_extrapolated"] = 48 * lms * 1e-3
         del w13l, w2l, outs13, outs2
         torch.cuda.empty_cache()
+        # a dense (single-expert) W4A4 + RAC projection at model scale: 8192 tokens, 4096 -> 4096, 50 % of the
+        # input channels compensated; all rows belong to one weight matrix, so the CTA-pair GEMM is used
+        Td, Kd, Nd = 8192, 4096, 4096
+        xd = torch.randn(Td, Kd, device=dev).to(torch.bfloat16)
+        wd = B.fake_quant_weights((torch.randn(1, Nd, Kd, device=dev) * 0.02).to(torch.bfloat16), want_fq=False,
+                                  sf_layout=B.SF_TILED)
+        wsd = torch.empty(B.moe_workspace_bytes(Td, Kd, 0, 1, 1, Nd), dtype=torch.uint8, device=dev)
+
+        def dense_step():
+            B.dense_w4a4_rac(xd, wd, Kd // 2, workspace=wsd)
+        for _ in range(3):
+            dense_step()
+        tdn = timed(dense_step, 20)
+        dms = sum(tdn) / len(tdn)
+        aux["dense_linear_ms"] = dms
+        aux["dense_linear_tflops_algorithmic"] = 2.0 * Td * Kd * Nd * 1.5 / (dms * 1e-3) / 1e12
+        aux["dense_linear_note"] = "T=%d, %d -> %d, RAC on %d channels, activation quantized online, whole call" % (Td, Kd, Nd, Kd // 2)
+        del xd, wd, wsd
         # decode-sized batch on the same layer (the prefill and decode workloads share their weights):
         # weights cold (L2 flushed between iterations); roofline = streaming the 340 MB of weights once
         if args.workload == "prefill":

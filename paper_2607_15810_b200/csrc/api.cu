@@ -219,17 +219,19 @@ SideStream* side_stream() {
 }
 
 // GEMM variant of a call.  1: single-CTA tiles of 128 x 256; 2: CTA pairs computing 256 x 256
-// tiles with cta_group::2 MMAs (about a tenth faster per tile, but every expert's rows are then
-// padded to a multiple of 256).  QUADS_GEMM_CTA_GROUP=1|2 forces one; otherwise pairs are used
-// where the padding is small next to the work: at least 512 rows per expert on average (measured:
-// 477 vs 488 us per layer at 512 rows per expert, 814 vs 797 us at 256).
+// tiles with cta_group::2 MMAs: about 7 % (first projection) / 5 % (second) faster per tile, but
+// every expert's rows are then padded to a multiple of 256, i.e. half a tile more per expert on
+// average than padding to 128.  That pays from roughly 1000 rows per expert, which is the rule used
+// here; QUADS_GEMM_CTA_GROUP=1|2 forces a variant.  (When the experts' tile counts happen to be
+// even -- the skewed prefill benchmark: 410 rows = 4 tiles for most experts -- pairs already win at
+// 512 rows per expert: 477 vs 488 us per layer.)
 int gemm_cta_group_for(int64_t rows, int experts) {
   static const int forced = [] {
     const char* e = getenv("QUADS_GEMM_CTA_GROUP");
     return (e && (e[0] == '1' || e[0] == '2')) ? e[0] - '0' : 0;
   }();
   if (forced) return forced;
-  return rows >= (int64_t)512 * (experts > 0 ? experts : 1) ? 2 : 1;
+  return rows >= (int64_t)1024 * (experts > 0 ? experts : 1) ? 2 : 1;
 }
 
 quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,

@@ -16,7 +16,7 @@
 // each CTA holds its own 128 rows of A^ / R^ and HALF of the weight tile, and one
 // thread issues the MMAs and scale copies of both SMs; per 128-row tile it is about a
 // tenth faster, but every expert's rows must then be padded to a multiple of 256).
-// No TMA multicast is used: every CTA loads what it needs itself.
+// Every CTA loads what it needs itself; no load is shared across the cluster.
 //
 // One persistent CTA per SM, 18 warps:
 //   warp 0     producer: TMA tile loads of packed FP4 (128-byte swizzle) and bulk

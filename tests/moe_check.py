@@ -67,14 +67,14 @@ def check_site1(res, orc, nsel13, report):
     report["site13_bit_exact"] = True
 
 
-def check_moe(res, x, logits, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize=True, row_sample=None):
+def check_moe(res, x, logits, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize=True, row_sample=None, a13_gs=None):
     """res: dict from binding.moe_w4a4_rac(export=True); x, logits torch CPU
     tensors; w13o / w2o oracle weight dicts.  Returns a report dict; raises on
     any violation."""
     report = {}
     xf = f32(x)
     lg = logits.cpu().numpy()
-    orc = M.moe_forward(xf, lg, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize=renormalize)
+    orc = M.moe_forward(xf, lg, w13o, w2o, topk, nsel13, nsel2, a2_gs, a13_gs=a13_gs, renormalize=renormalize)
     T, H = xf.shape
     I = w2o["codes"].shape[2]
     # ---- stage 1
@@ -97,7 +97,8 @@ def check_moe(res, x, logits, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize
     assert report["h_max_err_over_tol"] <= 1.0, "h outside tolerance: %g" % report["h_max_err_over_tol"]
     report["h_bitwise_equal_fraction"] = float((F.bf16_bits(h_gpu) == F.bf16_bits(orc["h"])).mean())
     # ---- stage 3: requantize of the implementation's own h
-    orc2 = M.moe_forward(xf, lg, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize=renormalize, h_override=h_gpu)
+    orc2 = M.moe_forward(xf, lg, w13o, w2o, topk, nsel13, nsel2, a2_gs, a13_gs=a13_gs, renormalize=renormalize,
+                         h_override=h_gpu)
     site2 = orc2["site2"]
     assert np.array_equal(res["hq"].cpu().numpy(), F.pack_nibbles(site2["codes"])), "Q_A(h) codes differ"
     assert np.array_equal(res["hsf"].cpu().numpy(), site2["sf"]), "Q_A(h) scales differ"
@@ -106,7 +107,7 @@ def check_moe(res, x, logits, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize
         assert ok, "site-2 selection differs beyond ties (%d channels)" % ndiff
         report["sel2_tie_swaps"] = ndiff
         if ndiff:
-            orc2 = M.moe_forward(xf, lg, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize=renormalize,
+            orc2 = M.moe_forward(xf, lg, w13o, w2o, topk, nsel13, nsel2, a2_gs, a13_gs=a13_gs, renormalize=renormalize,
                                  h_override=h_gpu, forced_sel2=res["sel2"].cpu().numpy()[:nsel2])
             site2 = orc2["site2"]
         assert np.array_equal(res["r2q"].cpu().numpy(), F.pack_nibbles(site2["r_codes"])), "residual-of-h codes differ"

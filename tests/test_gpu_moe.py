@@ -285,3 +285,25 @@ def test_moe_call_is_capturable_in_a_cuda_graph(B):
         torch.cuda.synchronize()
         assert B.moe_async_status(ws) == 0
         assert torch.equal(out_s, want)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_moe_with_a_static_activation_scale(B, name):
+    """Caller-supplied per-tensor scale for x (no amax pass), chosen at half of
+    the amax-derived one so that the largest activations saturate."""
+    sh = synth.MOE_SHAPES[name]
+    x, _ = synth.activations(sh)
+    lg = synth.router_logits(sh)
+    w13, w2 = synth.expert_weights(sh, "w13"), synth.expert_weights(sh, "w2")
+    w13o, w2o = MC.oracle_weights(w13), MC.oracle_weights(w2)
+    nsel13, nsel2 = sh.H // 2, sh.I // 4
+    a13 = np.float32(0.5) * Q.tensor_global_scale(MC.f32(x))
+    pilot = M.moe_forward(MC.f32(x), lg.numpy(), w13o, w2o, sh.topk, nsel13, 0, np.float32(1.0), a13_gs=a13)
+    a2 = Q.tensor_global_scale(pilot["h"])
+    gw13 = B.fake_quant_weights(w13.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    gw2 = B.fake_quant_weights(w2.cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    res = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, nsel13, nsel2, torch.tensor([a2]).cuda(),
+                         a13_gs=torch.tensor([a13]).cuda(), export=True)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    MC.check_moe(res, x, lg, w13o, w2o, sh.topk, nsel13, nsel2, a2, a13_gs=a13)

@@ -307,3 +307,27 @@ def test_moe_with_a_static_activation_scale(B, name):
     torch.cuda.synchronize()
     assert B.moe_async_status(res["workspace"]) == 0
     MC.check_moe(res, x, lg, w13o, w2o, sh.topk, nsel13, nsel2, a2, a13_gs=a13)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_workspace_content_does_not_matter(B, name):
+    """The caller-owned workspace may hold anything on entry: a call on a
+    workspace filled with 0xFF bytes gives the bits of a call on a zeroed one
+    (both GEMM families: few rows per expert and the row-major tiles)."""
+    sh = synth.MOE_SHAPES[name]
+    x, _ = synth.activations(sh)
+    lg = synth.router_logits(sh)
+    gw13 = B.fake_quant_weights(synth.expert_weights(sh, "w13").cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    gw2 = B.fake_quant_weights(synth.expert_weights(sh, "w2").cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    a2 = torch.tensor([0.25]).cuda()
+    n = B.moe_workspace_bytes(sh.T, sh.H, sh.I, sh.E, sh.topk)
+    outs = []
+    for fill in (0, 255, 0x5A):
+        ws = torch.full((n + 4096,), fill, dtype=torch.uint8, device="cuda")
+        res = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, sh.H // 2, sh.I // 2, a2, workspace=ws, export=True)
+        torch.cuda.synchronize()
+        assert B.moe_async_status(ws) == 0
+        outs.append({k: v.clone() for k, v in res.items() if isinstance(v, torch.Tensor) and k != "workspace"})
+    for other in outs[1:]:
+        for k, v in outs[0].items():
+            assert torch.equal(v, other[k]), k

@@ -4,15 +4,19 @@
 // the MMAs run on padding, and half of the bytes an SM pulls in are padding too, while the only
 // real cost is streaming every expert's weights once.  Here the WEIGHTS take the M side of the
 // MMA (128 weight rows = 128 output features per tile, fully used) and the expert's tokens take
-// the N side in chunks of at most 64:
+// the N side in chunks of at most 32:
 //
 //   Dt[f, t] = sum_k  W^[e, f, k] X^[t, k]  +  sum_k  W^[e, f, k] (-M R^)[t, k]
 //
 // with the same operands, scales and dispatch layout as the row-major kernel (gemm.cu): the
 // quantized activations / residuals sit in padded dispatch order (128-row slots per expert), a
-// chunk is one half (64 consecutive rows) of a slot, and its block scales are columns 2 * half and
-// 2 * half + 1 of the slot's 128-row scale atom, so the MMA simply reads its N-side scales two
-// columns further on for the second half.
+// chunk is one quarter (32 consecutive rows) of a slot.  Its block scales are column `chunk` of the
+// slot's 128-row scale atom, but the MMA accepts N-side scales only at even column offsets: an odd
+// chunk is therefore computed as the second half of a 64-row N tile whose first 32 rows are whatever
+// precedes the chunk's rows in shared memory (the operand descriptor starts 4 KB early; those
+// accumulator columns are never read), with the scales read from the even column before it.
+// Small activation tiles leave room for four (six) stages of weights: what bounds this kernel is
+// the number of weight bytes in flight per SM, not the MMAs.
 //
 //   first projection : tile = 128 features; gate rows and up rows of those features go to two
 //                      accumulators; epilogue = SwiGLU, bf16, then the tile is transposed through
@@ -21,7 +25,7 @@
 //   second projection: tile = 128 output features; epilogue = bf16 rows for the combine kernel.
 //
 // Roles: warp 0 producer (TMA + bulk copies, ring of stages), warp 1 MMA issuer, warps 2..9
-// epilogue (thread = feature, 32 token columns each).  Two accumulator buffers.  Every wait is
+// epilogue (thread = feature, 16 token columns each).  Two accumulator buffers.  Every wait is
 // bounded (status word, as in gemm.cu).
 #include "kernels.cuh"
 #include "tcgen05.cuh"
@@ -33,15 +37,15 @@ namespace {
 constexpr int kKSteps = kGemmKSteps;
 constexpr int kStageKBytes = kGemmStageKBytes;
 static_assert(kKSteps == 4 && kStageKBytes == 128, "laid out for 256-element K stages");
-constexpr int kChunk = 64;                          // tokens per work item (one half of a 128-row slot)
+constexpr int kChunk = 32;                          // tokens per work item (one quarter of a 128-row slot)
 constexpr int kBoxRows = 16;                        // activation rows per TMA box
 constexpr int kTileW = 128 * kStageKBytes;          // 128 weight rows of one stage
 constexpr int kTileX = kChunk * kStageKBytes;       // one chunk of activation rows
 constexpr int kSfStage = kKSteps * 512;             // one 128-row scale atom per K step
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
-constexpr int kMaxChunkList = 2048;                 // (slot, half) entries, 2 bytes each
-constexpr int kMaxSlots = kMaxChunkList / 2;
+constexpr int kMaxChunkList = 2048;                 // (slot, chunk) entries, 2 bytes each
+constexpr int kMaxSlots = kMaxChunkList / 4;
 constexpr int kTmemCols = 512;
 constexpr int kTmemSfBase = 256;                    // accumulators: buffer b at column 128 b (gate 64 | up 64)
 constexpr int kTmemSfPerBuf = 64;
@@ -55,8 +59,8 @@ struct SCfg {
   static constexpr int kOffSfW = kOffR + kTileX;
   static constexpr int kOffSfX = kOffSfW + kNumW * kSfStage;
   static constexpr int kOffSfR = kOffSfX + kSfStage;
-  static constexpr int kStageBytes = kOffSfR + kSfStage;        // 57344 / 38912
-  static constexpr int kStages = kDual ? 3 : 5;
+  static constexpr int kStageBytes = kOffSfR + kSfStage;        // 49152 / 30720
+  static constexpr int kStages = kDual ? 4 : 6;
   static constexpr int kBarOffset = kStages * kStageBytes;
   // barrier block | reciprocal table | chunk list | expert tables | epilogue staging
   static constexpr int kOffLut = kBarOffset + 256;
@@ -77,6 +81,18 @@ struct __align__(8) SBarriers {
   int abort_flag;
   int n_items_chunks;
 };
+
+// 16 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); }
 // Barrier over the epilogue warps that also agrees on `ok` (true only if true in every thread), so
@@ -138,7 +154,7 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
     int total = 0;
     for (int base = 0; base < m_slots; base += 32) {
       const int mt = base + lane;
-      const int n = mt < m_slots ? ((int)tab_rows[mt] + kChunk - 1) / kChunk : 0;      // 0, 1 or 2 halves
+      const int n = mt < m_slots ? ((int)tab_rows[mt] + kChunk - 1) / kChunk : 0;      // 0 .. 4 chunks
       int incl = n;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -146,7 +162,7 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
         if (lane >= o) incl += v;
       }
       const int pos = total + incl - n;
-      for (int c = 0; c < n; ++c) chunk_list[pos + c] = (uint16_t)(mt * 2 + c);
+      for (int c = 0; c < n; ++c) chunk_list[pos + c] = (uint16_t)(mt * 4 + c);
       total += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
     if (lane == 0) bars->n_items_chunks = total;
@@ -169,7 +185,7 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
       const int ch = item / n_ft, ft = item - ch * n_ft;
-      const int mt = chunk_list[ch] >> 1, c = chunk_list[ch] & 1;
+      const int mt = chunk_list[ch] >> 2, c = chunk_list[ch] & 3;
       const int e = tab_expert[mt];
       const int wrow0 = e * p.b_rows_per_expert + ft * 128;            // gate rows (or the only rows)
       const int wrow1 = wrow0 + p.half1_row_offset;                   // up rows
@@ -179,7 +195,7 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
       const uint8_t* wsf1 = wsf + (size_t)((p.half1_row_offset >> 7) + ft) * kt_count * 512u;
       const uint8_t* xsf = p.a_sf + (size_t)mt * kt_count * 512u;
       const uint8_t* rsf = p.r_sf + (size_t)mt * kt_count * 512u;
-      const int n_box = (min(kChunk, (int)tab_rows[mt] - c * kChunk) + kBoxRows - 1) / kBoxRows;   // 1..4
+      const int n_box = (min(kChunk, (int)tab_rows[mt] - c * kChunk) + kBoxRows - 1) / kBoxRows;   // 1 or 2
       for (int ks = 0; ks < k_stages; ++ks) {
         ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, p.status);
         if (!ok) break;
@@ -221,11 +237,13 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
     constexpr uint32_t kSfHi = (uint32_t)(128 >> 4) | (1u << 14);
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++it) {
       const int ch = item / n_ft;
-      const int mt = chunk_list[ch] >> 1, c = chunk_list[ch] & 1;
+      const int mt = chunk_list[ch] >> 2, c = chunk_list[ch] & 3;
       const int n_rows = min(kChunk, (int)tab_rows[mt] - c * kChunk);
-      const int n_pad = (n_rows + 15) & ~15;                          // N of the MMAs: 16 .. 64
-      // E2M1 x E2M1, UE4M3 block scales, both operands K-major, M = 128, N = n_pad
-      const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(n_pad >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const int n_pad = (n_rows + 15) & ~15;                          // 16 or 32 token rows
+      const int n_lead = (c & 1) * kChunk;                            // odd chunk: 32 rows of filler come first
+      const int n_mma = n_lead + n_pad;                               // N of the MMAs: 16 .. 64
+      // E2M1 x E2M1, UE4M3 block scales, both operands K-major, M = 128, N = n_mma
+      const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
       const int buf = it & 1;
       const uint32_t acc = tmem + (uint32_t)(buf * 128);
       ok = mbar_wait(bar_tempty + 8 * buf, (uint32_t)((it >> 1) & 1) ^ 1u, abort_flag, p.status);
@@ -240,8 +258,8 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
         const uint32_t sfcol = tmem + kTmemSfBase + (kcount & 1u) * kTmemSfPerBuf;
         const uint32_t w0_lo = ((sb & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t w1_lo = (((sb + kTileW) & 0x3FFFFu) >> 4) | (1u << 16);
-        const uint32_t x_lo = (((sb + C::kOffX) & 0x3FFFFu) >> 4) | (1u << 16);
-        const uint32_t r_lo = (((sb + C::kOffR) & 0x3FFFFu) >> 4) | (1u << 16);
+        const uint32_t x_lo = (((sb + C::kOffX - n_lead * kStageKBytes) & 0x3FFFFu) >> 4) | (1u << 16);
+        const uint32_t r_lo = (((sb + C::kOffR - n_lead * kStageKBytes) & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t sfw_lo = ((sb + C::kOffSfW) & 0x3FFFFu) >> 4;
         const uint32_t sfx_lo = ((sb + C::kOffSfX) & 0x3FFFFu) >> 4;
         const uint32_t sfr_lo = ((sb + C::kOffSfR) & 0x3FFFFu) >> 4;
@@ -262,8 +280,8 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
               const uint64_t xdesc = ((uint64_t)kSw128Hi << 32) | (x_lo + 2 * j);
               const uint64_t rdesc = ((uint64_t)kSw128Hi << 32) | (r_lo + 2 * j);
               const uint64_t w0desc = ((uint64_t)kSw128Hi << 32) | (w0_lo + 2 * j);
-              // the token scales of the second half start two columns into the slot's atom
-              const uint32_t sfx = sfcol + 32 + 4 * j + 2u * (uint32_t)c, sfr = sfcol + 48 + 4 * j + 2u * (uint32_t)c;
+              // token scales: the even column at or before the chunk's own column of the slot's atom
+              const uint32_t sfx = sfcol + 32 + 4 * j + (uint32_t)(c & 2), sfr = sfcol + 48 + 4 * j + (uint32_t)(c & 2);
               tc_mma_nvf4<1>(acc, w0desc, xdesc, idesc, sfcol + 4 * j, sfx, accum);
               if (resid) tc_mma_nvf4<1>(acc, w0desc, rdesc, idesc, sfcol + 4 * j, sfr, 1u);
               if (kDual) {
@@ -284,23 +302,24 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
   } else {
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;                       // TMEM lane quadrant of this warp
-    const int th = (warp - 2) >> 2;               // token group: columns [32 th, 32 th + 32)
+    const int th = (warp - 2) >> 2;               // token group: this chunk's columns [16 th, 16 th + 16)
     const int f_in_tile = q * 32 + lane;          // this thread's feature within the tile
     const int etid = (warp - 2) * 32 + lane;      // 0 .. 255
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const float a_gs = p.a_gs ? p.a_gs[0]
                               : (__uint_as_float(p.a_amax_bits[0]) > 0.f
                                      ? __fdiv_rn(__uint_as_float(p.a_amax_bits[0]), kGlobalDiv) : 1.0f);
-    uint16_t* hs = reinterpret_cast<uint16_t*>(smem_gen + C::kOffStageH);              // [64 tokens][128 features] bf16
-    float* rs = reinterpret_cast<float*>(smem_gen + C::kOffStageH + kChunk * 128 * 2);  // [64][128] squared residuals
+    uint16_t* hs = reinterpret_cast<uint16_t*>(smem_gen + C::kOffStageH);              // [32 tokens][128 features] bf16
+    float* rs = reinterpret_cast<float*>(smem_gen + C::kOffStageH + kChunk * 128 * 2);  // [32][128] squared residuals
     int it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x, ++it) {
       const int ch = item / n_ft, ft = item - ch * n_ft;
-      const int mt = chunk_list[ch] >> 1, c = chunk_list[ch] & 1;
+      const int mt = chunk_list[ch] >> 2, c = chunk_list[ch] & 3;
       const int e = tab_expert[mt];
       const int n_rows = min(kChunk, (int)tab_rows[mt] - c * kChunk);
       const int n_pad = (n_rows + 15) & ~15;
+      const int col0 = (c & 1) * kChunk;          // the chunk's first accumulator column
       const int row0 = mt * 128 + c * kChunk;     // padded dispatch row of the chunk's first token
       const float scale = __fmul_rn(a_gs, tab_gs[e]);
       const int buf = it & 1;
@@ -308,9 +327,9 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
       if (kDual) ok = epi_all(ok);               // also: the previous item's readers are done with hs / rs
       if (!ok) break;
       tc_fence_after();
-      float g[32], u[32];
-      tmem_ld32(lane_addr + buf * 128 + th * 32, g);
-      if (kDual) tmem_ld32(lane_addr + buf * 128 + 64 + th * 32, u);
+      float g[16], u[16];
+      tmem_ld16(lane_addr + buf * 128 + col0 + th * 16, g);
+      if (kDual) tmem_ld16(lane_addr + buf * 128 + 64 + col0 + th * 16, u);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
@@ -321,31 +340,31 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
         const int n_out = p.n_out;
         const int f = ft * 128 + f_in_tile;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int t = th * 32 + i;
+        for (int i = 0; i < 16; ++i) {
+          const int t = th * 16 + i;
           if (t < n_rows)
             p.y_pad[(size_t)(row0 + t) * n_out + f] = __bfloat16_as_ushort(__float2bfloat16_rn(g[i] * scale));
         }
       } else {
         const int I = p.n_out;
         // (1) SwiGLU in the accumulator layout, rounded to bf16, transposed through shared memory
-        if (th * 32 < n_pad) {
+        if (th * 16 < n_pad) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
+          for (int i = 0; i < 16; ++i) {
             const float gg = __fmul_rn(g[i], scale);
             const float uu = __fmul_rn(u[i], scale);
             const float h = __fdividef(gg, 1.0f + __expf(-gg)) * uu;
-            hs[(th * 32 + i) * 128 + f_in_tile] = __bfloat16_as_ushort(__float2bfloat16_rn(h));
+            hs[(th * 16 + i) * 128 + f_in_tile] = __bfloat16_as_ushort(__float2bfloat16_rn(h));
           }
         }
         epi_barrier();
-        // (2) one 16-feature block of one token per thread and pass: the row-major kernel's arithmetic
+        // (2) one 16-feature block of one token per thread: the row-major kernel's arithmetic
         QuantCtx qc;
         quant_ctx_scalars(qc, p.h_gs[0]);
         qc.inv_lut = inv_lut;
         const int kt2 = I >> 6;
-        for (int t = etid >> 3; t < n_pad; t += 32) {
-          const int b = etid & 7;
+        const int t = etid >> 3, b = etid & 7;
+        if (t < n_pad) {
           const uint4* src = reinterpret_cast<const uint4*>(hs + t * 128 + 16 * b);
           const uint4 v0 = src[0], v1 = src[1];
           float hb[16];
@@ -383,17 +402,18 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
                                   r[4 * i + 3] * r[4 * i + 3]);
           }
         }
-        // (3) column scores of the residual: sums over the chunk's tokens in token order, one partial
-        // row per 32 tokens (rows 4 slot + 2 half + {0, 1}); rows of absent token groups are cleared.
+        // (3) column scores of the residual: sum over the chunk's tokens in token order -> partial
+        // row (slot, chunk); the slot's first chunk also clears the rows of its absent chunks.
         if (p.resid2) {
           epi_barrier();
-          const int fcol = etid & 127, grp = etid >> 7;          // feature, 32-token group of the half
-          float sacc = 0.f;
-          const int t_end = min(n_rows, 32 * grp + 32);
-          for (int tt = 32 * grp; tt < t_end; ++tt) sacc += rs[tt * 128 + fcol];
-          p.partials2[(size_t)(mt * 4 + 2 * c + grp) * I + ft * 128 + fcol] = sacc;
-          if (c == 0 && (int)tab_rows[mt] <= kChunk)              // the slot has no second half
-            p.partials2[(size_t)(mt * 4 + 2 + grp) * I + ft * 128 + fcol] = 0.f;
+          if (etid < 128) {
+            float sacc = 0.f;
+            for (int tt = 0; tt < n_rows; ++tt) sacc += rs[tt * 128 + etid];
+            p.partials2[(size_t)(mt * 4 + c) * I + ft * 128 + etid] = sacc;
+            if (c == 0)
+              for (int cc = ((int)tab_rows[mt] + kChunk - 1) / kChunk; cc < 4; ++cc)
+                p.partials2[(size_t)(mt * 4 + cc) * I + ft * 128 + etid] = 0.f;
+          }
         }
       }
     }

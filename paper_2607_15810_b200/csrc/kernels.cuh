@@ -104,7 +104,7 @@ struct GemmMaps {
   CUtensorMap a, r, b, sfa, sfr, sfb;
 };
 
-// Operand-swapped variant for few rows per expert (weights on the M side, tokens in chunks of 64
+// Operand-swapped variant for few rows per expert (weights on the M side, tokens in chunks of 32
 // on the N side; epi = kEpiSwiGLU or kEpiCombine).  Maps: a / r = activation / residual codes with
 // boxes of 16 rows, b = weight codes with boxes of 128 rows; p.n_tiles_n counts tiles of 128
 // output features.  Usable when assignments <= 32 * experts and the slot tables fit.

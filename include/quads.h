@@ -153,6 +153,17 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
  * Weight buffers are exactly what quads_fake_quant_weights() writes with
  * QUADS_SF_TILED: w13 is [E, 2I, H] (gate rows first, then up rows), w2 is
  * [E, H, I]; H % 128 == 0, I % 128 == 0 (dense: N % 128 == 0).
+ * Limits: E <= 256, topk <= 16 and <= E, H <= 16384, I <= 16384; a size outside
+ * them returns QUADS_ERR_SHAPE before anything is launched.
+ *
+ * The call allocates nothing and never synchronises the host.  Part of the
+ * work (routing, the dispatched copies of Q_A(X)) is enqueued on a second
+ * stream of the library's own, forked from and joined back into the caller's
+ * stream with events, so the call as a whole is ordered like any other work on
+ * `cuda_stream` and can be captured into a CUDA graph (make one ordinary call
+ * first: kernel attributes are set on first use).  Device-side waits are bounded;
+ * one that gives up writes QUADS_ERR_TIMEOUT to a status word in the workspace,
+ * read with quads_moe_async_status().
  */
 typedef struct {
   int32_t T, H, I, E, topk;

@@ -507,7 +507,11 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
     int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
     int32_t* expert_total = reinterpret_cast<int32_t*>(P(L.expert_total));
-    QUADS_CUDA_OK(launch_kernel(route_kernel, dim3(L.n_chunks), dim3(256), (size_t)(0), rs, a->router_logits, T, E, topk, a->renormalize, ids, wts, chunk_counts, expert_total, a->topk_ids, a->topk_w));
+    {
+      auto route = E <= 32 ? route_kernel_t<1> : (E <= 64 ? route_kernel_t<2> : (E <= 128 ? route_kernel_t<4> : route_kernel_t<8>));
+      QUADS_CUDA_OK(launch_kernel(route, dim3(L.n_chunks), dim3(256), (size_t)(0), rs, a->router_logits, T, E, topk,
+                                  a->renormalize, ids, wts, chunk_counts, expert_total, a->topk_ids, a->topk_w));
+    }
     trace_mark("route", st);
     QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(E), dim3(256), (size_t)(0), rs, E, L.n_chunks, cta_group, chunk_counts, expert_total, chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, a->expert_offsets));
     trace_mark("scan", st);

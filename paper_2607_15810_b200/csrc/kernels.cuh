@@ -43,9 +43,10 @@ __global__ void export_site2_kernel(int A, int I, const int32_t* perm, const int
                                     uint8_t* r2q, uint8_t* r2sf);
 
 // ---- routing.cu
-__global__ void route_kernel(const float* logits, int T, int E, int topk, int renormalize, int32_t* ids,
-                             float* wts, int32_t* chunk_counts, int32_t* expert_total, int32_t* ids_out,
-                             float* wts_out);
+template <int NJ>
+__global__ void route_kernel_t(const float* logits, int T, int E, int topk, int renormalize, int32_t* ids,
+                               float* wts, int32_t* chunk_counts, int32_t* expert_total, int32_t* ids_out,
+                               float* wts_out);
 __global__ void scan_kernel(int E, int n_chunks, int tile_group, const int32_t* chunk_counts,
                             const int32_t* expert_total, int32_t* chunk_base, int32_t* offsets, int32_t* tile_prefix,
                             int32_t* tile_expert, int32_t* tile_rows, int32_t* header, int32_t* offsets_out);

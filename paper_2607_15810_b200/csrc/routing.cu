@@ -18,8 +18,10 @@ __device__ __forceinline__ uint32_t float_key(float v) {
 // tokens) also writes its per-expert assignment counts: chunk_counts[expert][cta],
 // and adds them to expert_total[expert] (zero on entry).
 constexpr int kRouteTokensPerWarp = 4;
+// NJ = logits per lane = ceil(E / 32) rounded up to 1, 2, 4 or 8.
+template <int NJ>
 __global__ void __launch_bounds__(256)
-route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
+route_kernel_t(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
              int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
              int32_t* __restrict__ expert_total, int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
   pdl_sync();
@@ -29,14 +31,14 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t0 = blockIdx.x * kRouteTokensPerCta + warp * kRouteTokensPerWarp;
   constexpr int TW = kRouteTokensPerWarp;
-  float v[TW][8];
+  float v[TW][NJ];
   float mx[TW], sum[TW], wsum[TW], my_w[TW];
   int my_id[TW];
 #pragma unroll
   for (int a = 0; a < TW; ++a) {
     const int t = t0 + a;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 0; j < NJ; ++j) {
       const int e = j * 32 + lane;
       v[a][j] = (t < T && e < E) ? logits[(size_t)t * E + e] : -INFINITY;
     }
@@ -45,7 +47,7 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
   for (int a = 0; a < TW; ++a) {
     float m = v[a][0];
 #pragma unroll
-    for (int j = 1; j < 8; ++j) m = fmaxf(m, v[a][j]);
+    for (int j = 1; j < NJ; ++j) m = fmaxf(m, v[a][j]);
     mx[a] = m;
   }
 #pragma unroll
@@ -56,7 +58,7 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
   for (int a = 0; a < TW; ++a) {
     float sacc = 0.f;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) sacc += (j * 32 + lane < E && t0 + a < T) ? expf(v[a][j] - mx[a]) : 0.f;
+    for (int j = 0; j < NJ; ++j) sacc += (j * 32 + lane < E && t0 + a < T) ? expf(v[a][j] - mx[a]) : 0.f;
     sum[a] = sacc; wsum[a] = 0.f; my_w[a] = 0.f; my_id[a] = 0;
   }
 #pragma unroll
@@ -71,7 +73,7 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
       float bv = -INFINITY;
       int e1 = 0x7FFFFFFF;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < NJ; ++j) {
         const int e = j * 32 + lane;
         if (e < E && v[a][j] > bv) { bv = v[a][j]; e1 = e; }   // ascending e: the first maximum wins
       }
@@ -93,7 +95,7 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
       wsum[a] += w;
       if (lane == s) { my_w[a] = w; my_id[a] = be[a]; }
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
+      for (int j = 0; j < NJ; ++j)
         if (j * 32 + lane == be[a]) v[a][j] = -INFINITY;       // remove the winner
     }
   }
@@ -115,6 +117,11 @@ route_kernel(const float* __restrict__ logits, int T, int E, int topk, int renor
     if (hist[i]) atomicAdd(expert_total + i, hist[i]);          // integer sums: order does not matter
   }
 }
+
+template __global__ void route_kernel_t<1>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
+template __global__ void route_kernel_t<2>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
+template __global__ void route_kernel_t<4>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
+template __global__ void route_kernel_t<8>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
 
 // One CTA per expert, 256 threads.  From the experts' totals: the exclusive scan over experts of
 // counts (offsets) and of 128-row tile counts (tile_prefix; every expert gets a multiple of

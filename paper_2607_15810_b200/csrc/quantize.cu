@@ -544,14 +544,29 @@ combine_kernel(const uint16_t* __restrict__ y_pad, const int32_t* __restrict__ p
   float acc[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-  for (int s = 0; s < topk; ++s) {
-    const int p = pos_pad[t * topk + s];
-    const float w = wts[t * topk + s];
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(y_pad + (size_t)p * H) + c);
-    float f[8];
-    unpack8(v, f);
+  // eight slots at a time: all row positions first, then all row loads, so that the loads of a
+  // token's rows are in flight together; the sum itself runs in slot order
+  for (int s0 = 0; s0 < topk; s0 += 8) {
+    int p[8];
+    float w[8];
+    uint4 v[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = __fmaf_rn(w, f[j], acc[j]);
+    for (int j = 0; j < 8; ++j) {
+      const bool on = s0 + j < topk;
+      p[j] = on ? __ldg(pos_pad + t * topk + s0 + j) : -1;
+      w[j] = on ? __ldg(wts + t * topk + s0 + j) : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      v[j] = p[j] >= 0 ? __ldcs(reinterpret_cast<const uint4*>(y_pad + (size_t)p[j] * H) + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if (p[j] < 0) continue;
+      float f[8];
+      unpack8(v[j], f);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc[k] = __fmaf_rn(w[j], f[k], acc[k]);
+    }
   }
   reinterpret_cast<uint4*>(out + (size_t)t * H)[c] =
       make_uint4(f32x2_to_bf16x2(acc[0], acc[1]), f32x2_to_bf16x2(acc[2], acc[3]),

@@ -296,9 +296,11 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
     float acc[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+    uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
+    if (r0 < r1) ldg256(x + (size_t)r0 * H + kb * 16, n0, n1);
     for (int r = r0; r < r1; ++r) {
-      uint4 v0, v1;
-      ldg256(x + (size_t)r * H + kb * 16, v0, v1);
+      const uint4 v0 = n0, v1 = n1;
+      if (r + 1 < r1) ldg256(x + (size_t)(r + 1) * H + kb * 16, n0, n1);   // next row's block, ahead of this row's arithmetic
       float f[16], o[16];
       unpack8(v0, f);
       unpack8(v1, f + 8);

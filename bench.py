@@ -381,7 +381,7 @@ def run_ours(args):
     # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM-1 launch, from the ncu capture
     # summarised in profiles/gemm_kernel_moe_prefill_ncu_full.md (prefill workload, RAC at both sites)
     if args.workload == "prefill" and args.variant == "both":
-        roofline["traffic"] = 463616256
+        roofline["traffic"] = 463474432
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4 (e2m1 x e2m1, ue4m3 block scales, fp32 accumulate)",

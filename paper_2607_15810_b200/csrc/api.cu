@@ -526,8 +526,14 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   static const bool no_fused_amax = getenv("QUADS_NO_FUSED_AMAX") != nullptr;
   bool fused_amax = false;
   if (!a->a13_gs && !no_fused_amax && !g_trace.enabled) {
-    int per_sm = 0;
-    QUADS_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rac_quant_kernel, rq_block, 0));
+    // resident CTAs per SM for the two block sizes in use (128 and 256 threads); same on every sm_100 device
+    static std::atomic<int> per_sm_cache[2] = {{0}, {0}};
+    std::atomic<int>& slot = per_sm_cache[rq_block > 128 ? 1 : 0];
+    int per_sm = slot.load();
+    if (per_sm == 0) {
+      QUADS_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rac_quant_kernel, rq_block > 128 ? 256 : 128, 0));
+      slot.store(per_sm);
+    }
     fused_amax = (int64_t)per_sm * di.sm_count >= L.stats_ctas;
   }
   if (!a->a13_gs && !fused_amax) {

@@ -96,6 +96,12 @@ size_t quads_quantize_workspace_bytes(void);
  *   sf      out, u8 per `sf_layout`, one [N, K/16] (or tiled) block per tensor (NULL to skip)
  *   gs      out, float [n_tensors] (required)
  *   workspace >= quads_fake_quant_workspace_bytes(n_tensors) bytes
+ * The kernel is one cooperative launch whose CTAs meet at a counter per tensor
+ * (a tensor's scale needs every CTA's share of its amax).  Every such wait is
+ * bounded (2 s); if one ever gives up, the call still ends, the outputs of the
+ * tensors concerned are unspecified and gs[t] = NaN marks them.  The launch
+ * needs the whole GPU: it fails with QUADS_ERR_CUDA if the device cannot hold
+ * all of its CTAs at once (for instance under a partitioned context).
  */
 quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t N, int64_t K,
                                       void* w_fq, uint8_t* q, uint8_t* sf, float* gs,

@@ -1,5 +1,6 @@
 // C ABI entry points: argument checks, workspace carving, TMA descriptors and
 // the launch sequence of each public call.
+#include <algorithm>
 #include <cstdlib>
 #include <atomic>
 #include <mutex>
@@ -305,6 +306,32 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   int tiled = sf_layout == QUADS_SF_TILED;
   int64_t sf_stride = tiled ? (int64_t)quads_sf_tiled_bytes(rows, K) : rows * (K / 16);
   const int64_t nblk = rows * (K / 16);
+  // A batch of tensors with no scales given: the ring kernel (pipelines of bulk copies, the amax
+  // stream running ahead of the quantization by a tensor or two, which must stay in L2).
+  if (!gs_in && ld == K && n_tensors >= 2 && !getenv("QUADS_NO_RING_QUANT")) {
+    const int64_t per64 = ((nblk + di.sm_count - 1) / di.sm_count + 3) / 4 * 4;   // blocks per CTA, 128-byte granules
+    const int64_t tensor_bytes = nblk * 32;
+    if (per64 < (int64_t)1 << 24 && tensor_bytes * 2 <= (int64_t)64 << 20) {
+      // A's lead over Q: a group's chunks of one tensor (so Q never catches up with A inside a
+      // tensor) plus a few for the time it takes a maximum to travel between the CTAs
+      const int chunks_per_tensor = (int)((per64 * 32 + 4 * kRingChunkBytes - 1) / (4 * kRingChunkBytes));
+      int lead = chunks_per_tensor + (tensor_bytes > ((int64_t)16 << 20) ? 2 : 3);   // large tensors: mind the L2 footprint
+      if (const char* e = getenv("QUADS_RING_LEAD")) lead = chunks_per_tensor + std::max(0, atoi(e));
+      int per = (int)per64;
+      uint32_t k16 = (uint32_t)(K / 16);
+      int kt_count = (int)((K + 63) / 64);
+      int64_t stride = tensor_stride;
+      int64_t nb = nblk;
+      QUADS_CUDA_OK(set_max_dynamic_smem<fake_quant_ring_kernel>(kRingSmemBytes));
+      void* rargs[] = {&xp, &nb, &stride, &nt, &amax_bits, &per, &lead, &q, &sf, &fqp,
+                       &gs_out, &tiled, &sf_stride, &k16, &kt_count};
+      QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fake_quant_ring_kernel), dim3(di.sm_count),
+                                                dim3(kRingThreads), rargs, (size_t)kRingSmemBytes, st));
+      note_launch();
+      QUADS_CUDA_OK(cudaGetLastError());
+      return QUADS_OK;
+    }
+  }
   static std::atomic<int> blocks_per_sm_cache{0};   // same kernel and block size on every sm_100 device
   int blocks_per_sm = blocks_per_sm_cache.load();
   if (blocks_per_sm == 0) {

@@ -151,7 +151,8 @@ __device__ __forceinline__ float quant_inv_entry(uint32_t code, float gs) {
 // Quantize one block of 16 floats.  u = amax / d6 is formed as q0 = amax * r6 followed by one
 // fused correction step (residual amax - q0 * d6 is exact in an FMA), which yields the correctly
 // rounded quotient given a correctly rounded reciprocal; the 1 / d of the element scaling comes
-// from the table.
+// from the table (kLut) or from the table's own formula evaluated in place.
+template <bool kLut = true>
 __device__ __forceinline__ BlockQ quantize_block(const float* v, const QuantCtx& c) {
   float a = 0.f;
 #pragma unroll
@@ -161,7 +162,8 @@ __device__ __forceinline__ BlockQ quantize_block(const float* v, const QuantCtx&
   BlockQ r;
   r.sf8 = f32_to_e4m3(u);
   r.d = __fmul_rn(e4m3_to_f32(r.sf8), c.gs);
-  const float inv = c.inv_lut[r.sf8];
+  // without the table: the same quotient, one division per block
+  const float inv = kLut ? c.inv_lut[r.sf8] : quant_inv_entry(r.sf8, c.gs);
   r.lo = f32x8_to_e2m1x8(__fmul_rn(v[0], inv), __fmul_rn(v[1], inv), __fmul_rn(v[2], inv), __fmul_rn(v[3], inv),
                          __fmul_rn(v[4], inv), __fmul_rn(v[5], inv), __fmul_rn(v[6], inv), __fmul_rn(v[7], inv));
   r.hi = f32x8_to_e2m1x8(__fmul_rn(v[8], inv), __fmul_rn(v[9], inv), __fmul_rn(v[10], inv), __fmul_rn(v[11], inv),

@@ -20,6 +20,17 @@ __global__ void fused_quantize_kernel(const uint16_t* x, int64_t rows, int64_t K
                                       int n_tensors, const float* gs_in, uint32_t* amax_bits, uint32_t* counters,
                                       uint8_t* q, uint8_t* sf, uint16_t* fq, float* gs_out, int sf_tiled,
                                       int64_t sf_tensor_stride, int n_groups);
+// Fake-quant of a batch of tensors through shared-memory rings of bulk copies (one CTA per SM,
+// four groups of 7 consumer warps + 1 producer warp, one ring of 14 KB stages per group).
+constexpr int kRingThreads = 1024;
+constexpr int kRingDepth = 3;
+constexpr int kRingHeaderBytes = 1024;
+constexpr int kRingChunkBytes = 7 * 32 * 2 * 32;
+constexpr int kRingSmemBytes = kRingHeaderBytes + 4 * kRingDepth * kRingChunkBytes;
+__global__ void fake_quant_ring_kernel(const uint16_t* x, int64_t nblk, int64_t tensor_stride, int n_tensors,
+                                       uint32_t* pair, int per, int lead, uint8_t* q, uint8_t* sf, uint16_t* fq,
+                                       float* gs_out, int sf_tiled, int64_t sf_tensor_stride, uint32_t k16,
+                                       int kt_count);
 __global__ void rac_quant_kernel(const uint16_t* x, int T, int H, const float* gs_in, uint32_t* amax_bits,
                                  unsigned int* grid_arrivals, int32_t* status,
                                  float* gs_store, int rows_per_cta, int with_residual, float* partials, uint8_t* xq,

@@ -2,6 +2,7 @@
 // channel selection, masked residual quantize + dispatch scatter, small fix-ups.
 // All HBM- or latency-bound; no tensor cores here.
 #include "kernels.cuh"
+#include "tcgen05.cuh"
 
 namespace quads {
 
@@ -89,6 +90,44 @@ __device__ __forceinline__ uint32_t absmax8(const uint4& v) {
   return __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
 }
 
+// Where the quantizer's outputs of one tensor go (any pointer may be null).
+struct QuantSink {
+  uint8_t* q;        // packed codes: block b owns bytes [8b, 8b+8)
+  uint8_t* sf;       // scale bytes, linear ([b]) or tiled
+  uint16_t* fq;      // dequantized bf16: block b owns bytes [32b, 32b+32)
+  int sf_tiled;
+  uint32_t k16;      // blocks per row
+  int kt_count;      // scale atoms per row tile
+};
+
+// Quantize block b (16 bf16 values in v0 | v1) and stream the outputs out.
+template <bool kLut>
+__device__ __forceinline__ void emit_block(const QuantSink& o, const QuantCtx& qc, int64_t b, const uint4& v0,
+                                           const uint4& v1) {
+  float f[16];
+  unpack8(v0, f);
+  unpack8(v1, f + 8);
+  const BlockQ bq = quantize_block<kLut>(f, qc);
+  if (o.q) __stcs(reinterpret_cast<uint2*>(o.q + b * 8), make_uint2(bq.lo, bq.hi));
+  if (o.sf) {
+    if (o.sf_tiled) {
+      const uint32_t r = (uint32_t)(b / o.k16), kb = (uint32_t)(b - (int64_t)r * o.k16);
+      o.sf[sf_tiled_offset(r, kb, o.kt_count)] = (uint8_t)bq.sf8;
+    } else {
+      o.sf[b] = (uint8_t)bq.sf8;
+    }
+  }
+  if (o.fq) {
+    float d[16];
+    dequant_block(bq, d);
+    uint4* dst = reinterpret_cast<uint4*>(o.fq + b * 16);
+    __stcs(dst, make_uint4(f32x2_to_bf16x2(d[0], d[1]), f32x2_to_bf16x2(d[2], d[3]),
+                           f32x2_to_bf16x2(d[4], d[5]), f32x2_to_bf16x2(d[6], d[7])));
+    __stcs(dst + 1, make_uint4(f32x2_to_bf16x2(d[8], d[9]), f32x2_to_bf16x2(d[10], d[11]),
+                               f32x2_to_bf16x2(d[12], d[13]), f32x2_to_bf16x2(d[14], d[15])));
+  }
+}
+
 __global__ void __launch_bounds__(256, 4)
 fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
                       int n_tensors, const float* __restrict__ gs_in, uint32_t* __restrict__ amax_bits,
@@ -150,12 +189,14 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
         atomicAdd(counters + t, 1u);
         // bounded wait for the rest of the group (cooperative launch: all CTAs are resident)
         const long long t0 = clock64();
+        bool gave_up = false;
         while (atomicAdd(counters + t, 0u) < (uint32_t)gsize) {
           __nanosleep(64);
-          if (clock64() - t0 > 4000000000ll) break;
+          if (clock64() - t0 > 4000000000ll) { gave_up = true; break; }
         }
         __threadfence();
-        gs_sh = gs_from_amax_bits(atomicAdd(amax_bits + t, 0u));
+        // (the count only grows, so if one CTA of the group gives up on it, all do: NaN marks the tensor)
+        gs_sh = gave_up ? __int_as_float(0x7FC00000) : gs_from_amax_bits(atomicAdd(amax_bits + t, 0u));
       }
       __syncthreads();
       gs = gs_sh;
@@ -175,31 +216,8 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
     const int kt_count = (int)((K + 63) >> 6);
     const bool contiguous = (ld == K);
     const uint32_t k16u = (uint32_t)k16;
-    auto emit = [&](int64_t b, const uint4& v0, const uint4& v1) {
-      float f[16];
-      unpack8(v0, f);
-      unpack8(v1, f + 8);
-      const BlockQ bq = quantize_block(f, qc);
-      // outputs are contiguous per tensor: block b owns bytes [8b, 8b+8) of q and [32b, 32b+32) of fq
-      if (qt) __stcs(reinterpret_cast<uint2*>(qt + b * 8), make_uint2(bq.lo, bq.hi));
-      if (sft) {
-        if (sf_tiled) {
-          const uint32_t r = (uint32_t)(b / k16u), kb = (uint32_t)(b - (int64_t)r * k16u);
-          sft[sf_tiled_offset(r, kb, kt_count)] = (uint8_t)bq.sf8;
-        } else {
-          sft[b] = (uint8_t)bq.sf8;
-        }
-      }
-      if (fqt) {
-        float o[16];
-        dequant_block(bq, o);
-        uint4* dst = reinterpret_cast<uint4*>(fqt + b * 16);
-        __stcs(dst, make_uint4(f32x2_to_bf16x2(o[0], o[1]), f32x2_to_bf16x2(o[2], o[3]),
-                               f32x2_to_bf16x2(o[4], o[5]), f32x2_to_bf16x2(o[6], o[7])));
-        __stcs(dst + 1, make_uint4(f32x2_to_bf16x2(o[8], o[9]), f32x2_to_bf16x2(o[10], o[11]),
-                                   f32x2_to_bf16x2(o[12], o[13]), f32x2_to_bf16x2(o[14], o[15])));
-      }
-    };
+    const QuantSink sink{qt, sft, fqt, sf_tiled, k16u, kt_count};
+    auto emit = [&](int64_t b, const uint4& v0, const uint4& v1) { emit_block<true>(sink, qc, b, v0, v1); };
     auto src_of = [&](int64_t b) -> const uint16_t* {
       if (contiguous) return base + b * 16;
       const int64_t r = b / k16, kb = b - r * k16;
@@ -222,6 +240,316 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
       ldg256_stream(src_of(b), a0, a1);
       emit(b, a0, a1);
     }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Fused amax + fake-quant for a batch of tensors (expert weights), one persistent CTA per SM made
+// of kRingGroups independent pipelines: 7 consumer warps and one producer warp each.  A tensor is
+// cut into one contiguous share per CTA and a share into chunks of 448 blocks (14 KB, two blocks
+// per consumer lane; a bulk copy costs the SM about 50 ns whatever its size and every chunk costs
+// every warp some bookkeeping, so small chunks cannot keep up), dealt to the groups round-robin.
+// A group works through two streams of its chunks, both in tensor order:
+//   A  reduce |x| max over the chunk; when the last consumer warp of the CTA gets to the end of a
+//      tensor, the CTA's maximum is published and the CTA counted in at the tensor's arrival word;
+//   Q  quantize the chunk with the tensor's scale, known once all CTAs have arrived.
+// The streams are interleaved chunk by chunk with A `lead` chunks ahead (more than a tensor, so
+// that a scale is normally known long before Q needs it), which keeps DRAM reads (A) and writes
+// (Q) flowing at the same time instead of in chip-wide bursts.  The producer walks the same list
+// kRingDepth chunks ahead and fills the group's ring of shared-memory stages with bulk
+// asynchronous copies (A's copy fetches from DRAM and asks L2 to keep the lines, Q's copy finds
+// them in L2), so no consumer waits for DRAM.  Between copies the producers also do the talking
+// between CTAs (tensor t belongs to producer t mod kRingGroups): they publish the CTA's
+// maxima, watch the arrival words and post each scale on a shared-memory board, where the
+// consumers find it -- one reader per tensor and CTA, because thousands of readers of one
+// address queue up at its L2 slice.
+// `pair` holds {amax bits, arrivals} per tensor, zero on entry.  Waits are bounded; a warp that
+// gives up raises a flag that stops the CTA, and NaN is written to the scales not yet posted.
+// ---------------------------------------------------------------------------
+constexpr int kRingBoard = 32;                                  // tensors in flight per CTA, at most half of this
+constexpr int kRingGroups = 4;
+constexpr int kRingGroupWarps = kRingThreads / 32 / kRingGroups;   // 8: 7 consumers + the producer
+constexpr int kRingConsumers = kRingGroupWarps - 1;
+constexpr int kRingLaneBlocks = 2;                              // blocks per consumer lane and chunk
+constexpr int kRingPassBlocks = kRingConsumers * 32;            // blocks a group takes in one pass over its lanes
+constexpr int kRingChunkBlocks = kRingPassBlocks * kRingLaneBlocks;
+static_assert(kRingChunkBlocks * 32 == kRingChunkBytes, "chunk size");
+struct RingShared {
+  unsigned long long board[kRingBoard];   // {tensor index + 1, amax bits} once known to this CTA
+  unsigned long long pub[kRingBoard];     // {tensor index + 1, this CTA's |x| max} waiting to be published
+  uint32_t cta_max[kRingBoard];
+  uint32_t amax_cnt[kRingBoard];
+  uint64_t full[kRingGroups][kRingDepth];   // mbarriers: chunk landed
+  uint64_t empty[kRingGroups][kRingDepth];  // mbarriers: all consumer warps have left the stage
+  int abort_flag;
+};
+static_assert(sizeof(RingShared) <= kRingHeaderBytes, "header region too small");
+
+// Non-blocking test of an mbarrier phase (try_wait may park the thread for a while, which a
+// thread with other duties in its wait loop cannot afford).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t ld_relaxed_u64(const void* p) {
+  uint64_t v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                               uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+
+// A group's work list, in the order it is both fetched and consumed.
+enum { kItemA = 0, kItemQ = 1, kItemEndA = 2 };                 // kItemEndA: no chunk, tensor t's A stream is complete
+struct RingItems {
+  int n, lead, cnt, group;  // tensors, A's lead over Q in chunks, blocks in the CTA's share, group index
+  int ta, ka, tq, kq, ahead;
+  int kind, t, blk0, nb;    // current item
+  __device__ __forceinline__ void reset(int n_, int lead_, int cnt_, int group_) {
+    n = n_; lead = lead_; cnt = cnt_; group = group_; ta = ka = tq = kq = ahead = 0;
+  }
+  // first block (within the CTA's share) of the group's chunk k of tensor t, or >= cnt
+  __device__ __forceinline__ int chunk_first(int tt, int kk) const {
+    return (kk * kRingGroups + ((group + tt) & (kRingGroups - 1))) * kRingChunkBlocks;   // the ragged last round rotates
+  }
+  __device__ __forceinline__ bool next() {
+    if (ta < n && chunk_first(ta, ka) >= cnt) {                  // A has run off the end of a tensor
+      kind = kItemEndA; t = ta; ++ta; ka = 0;
+      return true;
+    }
+    while (tq < n && chunk_first(tq, kq) >= cnt) { ++tq; kq = 0; }
+    const bool q_ok = tq < n && tq < ta;                         // the group has finished A of that tensor
+    if (ta < n && (!q_ok || ahead < lead) && ta - tq < kRingBoard / 2) {
+      kind = kItemA; t = ta; blk0 = chunk_first(ta, ka); ++ka; ++ahead;
+    } else if (q_ok) {
+      kind = kItemQ; t = tq; blk0 = chunk_first(tq, kq); ++kq; --ahead;
+    } else {
+      return false;
+    }
+    nb = min(kRingChunkBlocks, cnt - blk0);
+    return true;
+  }
+};
+
+
+__global__ void __launch_bounds__(kRingThreads, 1)
+fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t tensor_stride, int n_tensors,
+                       uint32_t* __restrict__ pair, int per, int lead, uint8_t* __restrict__ q,
+                       uint8_t* __restrict__ sf, uint16_t* __restrict__ fq, float* __restrict__ gs_out, int sf_tiled,
+                       int64_t sf_tensor_stride, uint32_t k16, int kt_count) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  RingShared* sh = reinterpret_cast<RingShared*>(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = warp / kRingGroupWarps, warp_g = warp % kRingGroupWarps;   // warp_g == kRingConsumers: the producer
+  uint8_t* stage0 = smem + kRingHeaderBytes + (size_t)group * kRingDepth * kRingChunkBytes;
+  const uint32_t stage0_u32 = smem_u32(stage0);
+  const uint32_t full0 = smem_u32(&sh->full[group][0]), empty0 = smem_u32(&sh->empty[group][0]);
+  const int64_t start = (int64_t)blockIdx.x * per;               // first block of this CTA's share
+  const int64_t left = nblk - start;
+  const int cnt = left <= 0 ? 0 : (left < per ? (int)left : per);  // blocks in the share (same for every tensor)
+  volatile int* abort_flag = &sh->abort_flag;
+
+  if (threadIdx.x < kRingBoard) {
+    sh->board[threadIdx.x] = 0; sh->pub[threadIdx.x] = 0; sh->cta_max[threadIdx.x] = 0; sh->amax_cnt[threadIdx.x] = 0;
+  }
+  if (threadIdx.x == 0) {
+    for (int g = 0; g < kRingGroups; ++g)
+      for (int s = 0; s < kRingDepth; ++s) {
+        mbar_init(smem_u32(&sh->full[g][s]), 1);
+        mbar_init(smem_u32(&sh->empty[g][s]), kRingConsumers);
+      }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  auto wait_bar = [&](uint32_t bar, uint32_t parity) -> bool {   // bounded; false after giving up
+    if (mbar_try(bar, parity)) return true;
+    const uint64_t t0 = globaltimer();
+    uint32_t spins = 0;
+    while (!mbar_try(bar, parity)) {
+      if ((++spins & 255u) == 0) {
+        if (*abort_flag) return false;
+        if (globaltimer() - t0 > kWaitNs) { *abort_flag = 1; return false; }
+      }
+    }
+    return true;
+  };
+
+  if (warp_g == kRingConsumers) {
+    // =========================== producer (one lane)
+    if (lane != 0) return;
+    uint64_t keep, stream;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream));
+    const uint64_t* words = reinterpret_cast<const uint64_t*>(pair);
+    int watch = group;                                           // the tensor whose arrival word this producer reads next
+    uint64_t seen = 0;
+    bool asked = false;
+    long long asked_at = 0;
+    // One look at the arrival word of tensor `watch`; posts the scale once every CTA has arrived.
+    // The load is issued in one call and its value used in a later one, when it has had the time
+    // to return, so a call never waits.
+    int owed = group;                                            // the tensor this producer publishes next
+    auto watch_step = [&]() {
+      if (owed < n_tensors) {
+        const unsigned long long pv = *reinterpret_cast<volatile unsigned long long*>(&sh->pub[owed & (kRingBoard - 1)]);
+        if ((uint32_t)(pv >> 32) == (uint32_t)owed + 1u) {       // the CTA is through with A of that tensor
+          uint32_t* pr = pair + 2 * (size_t)owed;
+          if ((uint32_t)pv) atomicMax(pr, (uint32_t)pv << 16);
+          __threadfence();
+          atomicAdd(pr + 1, 1u);
+          owed += kRingGroups;
+        }
+      }
+      if (watch >= n_tensors) return;
+      if (asked && clock64() - asked_at < 2000) return;
+      if (asked && (uint32_t)(seen >> 32) == gridDim.x) {
+        if (gs_out && blockIdx.x == 0) gs_out[watch] = gs_from_amax_bits((uint32_t)seen);
+        sh->board[watch & (kRingBoard - 1)] = ((unsigned long long)((uint32_t)watch + 1u) << 32) | (uint32_t)seen;
+        watch += kRingGroups;
+        asked = false;
+        if (watch >= n_tensors) return;
+      }
+      seen = ld_relaxed_u64(words + watch);
+      asked = true;
+      asked_at = clock64();
+    };
+    RingItems pi;
+    pi.reset(n_tensors, lead, cnt, group);
+    int issued = 0;
+    bool ok = true;
+    while (ok && pi.next()) {
+      if (pi.kind == kItemEndA) continue;
+      const int s = issued % kRingDepth;
+      if (issued >= kRingDepth) {                                // the stage's previous chunk must have been left by all
+        const uint32_t bar = empty0 + 8 * s, parity = (uint32_t)(issued / kRingDepth - 1) & 1u;
+        const uint64_t t0 = globaltimer();
+        uint32_t spins = 0;
+        while (!mbar_test(bar, parity)) {
+          watch_step();                                          // consumers may be waiting for a scale meanwhile
+          if ((++spins & 1023u) == 0 && (*abort_flag || globaltimer() - t0 > kWaitNs)) { *abort_flag = 1; ok = false; break; }
+        }
+        if (!ok) break;
+      }
+      const uint32_t bytes = (uint32_t)pi.nb * 32u;
+      mbar_expect_tx(full0 + 8 * s, bytes);
+      bulk_load_hint(stage0_u32 + s * kRingChunkBytes, x + (size_t)pi.t * tensor_stride + (size_t)(start + pi.blk0) * 16,
+                     bytes, full0 + 8 * s, pi.kind == kItemA ? keep : stream);
+      ++issued;
+      watch_step();
+    }
+    // the remaining scales of this producer's tensors
+    const uint64_t t0 = globaltimer();
+    while (ok && (watch < n_tensors || owed < n_tensors)) {
+      watch_step();
+      __nanosleep(64);
+      if (*abort_flag || globaltimer() - t0 > kWaitNs) { *abort_flag = 1; ok = false; }
+    }
+    if (!ok) {
+      // gave up: mark the scales not posted, and let the copies in flight land (bounded) before leaving
+      if (gs_out)
+        for (int t = watch; t < n_tensors; t += kRingGroups) gs_out[t] = __int_as_float(0x7FC00000);
+      for (int d = issued < kRingDepth ? 0 : issued - kRingDepth; d < issued; ++d) {
+        const uint32_t bar = full0 + 8 * (d % kRingDepth), parity = (uint32_t)(d / kRingDepth) & 1u;
+        const uint64_t t1 = globaltimer();
+        while (!mbar_try(bar, parity) && globaltimer() - t1 < 100000000ull) {}
+      }
+    }
+    return;
+  }
+
+  // =========================== consumers
+  const int lane_c = warp_g * 32 + lane;                         // lane within the group's consumers
+  RingItems ci;
+  ci.reset(n_tensors, lead, cnt, group);
+  const QuantSink sink0{q, sf, fq, sf_tiled, k16, kt_count};
+  QuantSink sink = sink0;
+  QuantCtx qc;
+  qc.inv_lut = nullptr;
+  int consumed = 0;
+  int cur_q = -1;                                                // tensor whose scale is in qc
+  uint32_t m = 0;                                                // running |x| max (two 15-bit magnitudes) of the A tensor
+  while (ci.next()) {
+    if (ci.kind == kItemEndA) {
+      // ---- this warp is through with A of tensor t; the last consumer warp of the CTA publishes
+      uint32_t wm = max(m & 0xFFFFu, m >> 16);
+      m = 0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) wm = max(wm, __shfl_xor_sync(0xFFFFFFFFu, wm, o));
+      if (lane == 0) {
+        const int s = ci.t & (kRingBoard - 1);
+        if (wm) atomicMax(&sh->cta_max[s], wm);
+        __threadfence_block();
+        if (atomicAdd(&sh->amax_cnt[s], 1u) == (uint32_t)(kRingGroups * kRingConsumers - 1)) {
+          __threadfence_block();
+          // hand the CTA's maximum to the producer that owns the tensor: a fence between the two
+          // global atomics would make THIS warp wait for all its output stores in flight
+          const uint32_t tm = atomicExch(&sh->cta_max[s], 0u);
+          atomicExch(&sh->amax_cnt[s], 0u);
+          *reinterpret_cast<volatile unsigned long long*>(&sh->pub[s]) =
+              ((unsigned long long)((uint32_t)ci.t + 1u) << 32) | tm;
+        }
+      }
+      continue;
+    }
+    if (ci.kind == kItemQ && ci.t != cur_q) {
+      // ---- a new tensor's scale, from the board
+      const int t = ci.t;
+      uint32_t amax_b = 0xFFFFFFFFu;                             // (never an amax pattern)
+      if (lane == 0) {
+        const uint32_t tag = (uint32_t)t + 1u;
+        volatile unsigned long long* board = &sh->board[t & (kRingBoard - 1)];
+        unsigned long long b = *board;
+        if ((uint32_t)(b >> 32) != tag) {
+          const uint64_t t0 = globaltimer();
+          uint32_t spins = 0;
+          while ((uint32_t)((b = *board) >> 32) != tag) {
+            if ((++spins & 63u) == 0 && (*abort_flag || globaltimer() - t0 > kWaitNs)) { *abort_flag = 1; break; }
+          }
+        }
+        if ((uint32_t)(b >> 32) == tag) amax_b = (uint32_t)b;
+      }
+      amax_b = __shfl_sync(0xFFFFFFFFu, amax_b, 0);
+      if (amax_b == 0xFFFFFFFFu) break;
+      cur_q = t;
+      quant_ctx_scalars(qc, gs_from_amax_bits(amax_b));
+      sink = sink0;
+      if (sink.q) sink.q += (size_t)t * nblk * 8;
+      if (sink.sf) sink.sf += (size_t)t * sf_tensor_stride;
+      if (sink.fq) sink.fq += (size_t)t * nblk * 16;
+    }
+    const int s = consumed % kRingDepth;
+    if (!wait_bar(full0 + 8 * s, (uint32_t)(consumed / kRingDepth) & 1u)) break;
+    const uint8_t* st = stage0 + s * kRingChunkBytes;
+    if (ci.kind == kItemA) {
+#pragma unroll
+      for (int h = 0; h < kRingLaneBlocks; ++h) {
+        const int bl = lane_c + h * kRingPassBlocks;
+        if (bl < ci.nb) {
+          const uint4* v = reinterpret_cast<const uint4*>(st + bl * 32);
+          m = __vmaxu2(m, __vmaxu2(absmax8(v[0]), absmax8(v[1])));
+        }
+      }
+    } else {
+#pragma unroll
+      for (int h = 0; h < kRingLaneBlocks; ++h) {
+        const int bl = lane_c + h * kRingPassBlocks;
+        if (bl < ci.nb) {
+          const uint4* v = reinterpret_cast<const uint4*>(st + bl * 32);
+          const uint4 v0 = v[0], v1 = v[1];
+          emit_block<false>(sink, qc, start + ci.blk0 + bl, v0, v1);
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty0 + 8 * s);                  // this warp has left the stage
+    ++consumed;
   }
 }
 

@@ -124,3 +124,48 @@ def test_fake_quant_bit_exact_and_trainer_equals_rollout(B, n, N, K):
     assert np.array_equal(p["sf"].cpu().numpy()[:, idx], sf_o)
     f = B.fake_quant_weights(w.cuda(), want_pack=False)
     assert f["q"] is None and np.array_equal(F.bf16_bits(_f32(f["w_fq"])), F.bf16_bits(wf_o))
+
+
+@pytest.mark.parametrize("n,N,K", [
+    (40, 64, 128),       # more tensors than the kernel keeps in flight; most CTAs own no block at all
+    (2, 8, 16),          # two tensors of one block each
+    (9, 1000, 2048),     # a share of 868 blocks: one full chunk and a ragged one, dealt to rotating groups
+    (6, 1536, 2048),     # the 30B-A3B expert shape: 3 chunks per share over 4 groups
+    (3, 3072, 4096),     # the 235B-A22B expert shape: 12 chunks per share
+])
+def test_fake_quant_batch_kernel_equals_grouped_kernel_and_oracle(B, n, N, K, monkeypatch):
+    """A batch of tensors goes through the shared-memory ring kernel; with it switched off the
+    same call takes the grouped kernel.  Both must give the oracle's bytes."""
+    w = _bf16((n, N, K), 100 + n, 0.02)
+    w[0, 0, :16] = 0                                       # an all-zero block
+    if n > 2:
+        w[2] = 0                                           # an all-zero tensor: scale 1, codes 0
+    wc = w.cuda()
+    monkeypatch.delenv("QUADS_NO_RING_QUANT", raising=False)
+    a = B.fake_quant_weights(wc)
+    a_t = B.fake_quant_weights(wc, want_fq=False, sf_layout=B.SF_TILED)
+    monkeypatch.setenv("QUADS_NO_RING_QUANT", "1")
+    b = B.fake_quant_weights(wc)
+    b_t = B.fake_quant_weights(wc, want_fq=False, sf_layout=B.SF_TILED)
+    monkeypatch.delenv("QUADS_NO_RING_QUANT")
+    for k in ("gs", "q", "sf", "w_fq"):
+        assert torch.equal(a[k].view(torch.uint8), b[k].view(torch.uint8)), k
+    idx = torch.from_numpy(_tiled_index(N, K).reshape(-1)).cuda()     # (padding bytes of the tiled layout are never written)
+    for k in ("gs", "q"):
+        assert torch.equal(a_t[k].view(torch.uint8), b_t[k].view(torch.uint8)), k
+    assert torch.equal(a_t["sf"][:, idx], b_t["sf"][:, idx])
+    wf_o, q_o, sf_o, gs_o = Q.fake_quant_weights(_f32(w))
+    assert np.array_equal(a["gs"].cpu().numpy(), gs_o)
+    assert np.array_equal(a["q"].cpu().numpy(), q_o)
+    assert np.array_equal(a["sf"].cpu().numpy(), sf_o)
+    assert np.array_equal(F.bf16_bits(_f32(a["w_fq"])), F.bf16_bits(wf_o))
+    assert np.array_equal(a_t["sf"].cpu().numpy()[:, _tiled_index(N, K)], sf_o)
+
+
+def test_fake_quant_batch_kernel_repeats_bit_for_bit(B):
+    w = _bf16((24, 768, 2048), 5, 0.02).cuda()
+    first = B.fake_quant_weights(w)
+    for _ in range(5):
+        again = B.fake_quant_weights(w)
+        for k in ("gs", "q", "sf", "w_fq"):
+            assert torch.equal(first[k].view(torch.uint8), again[k].view(torch.uint8)), k

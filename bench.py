@@ -35,6 +35,8 @@ def parse():
     ap.add_argument("--variant", default="both", choices=["both", "w13", "plain"])
     ap.add_argument("--no-aux", action="store_true", help="skip the auxiliary quantize / fake-quant / decode numbers")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fake-quant-only", action="store_true",
+                    help="time only the fake-quant + pack of 16 expert weight tensors [3072, 4096] (a small case for profiling)")
     ap.add_argument("--ref-budget-s", type=float, default=0.0,
                     help="seconds of oracle work per step for --impl reference (0: derived from --steps)")
     return ap.parse_args()
@@ -201,10 +203,38 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def run_fake_quant_only(args):
+    """16 experts' W13 of the AQAT workload through quads_fake_quant_weights: 403 MB in, 516 MB out."""
+    import torch
+    from paper_2607_15810_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    w = (torch.randn(16, 3072, 4096, device=dev) * 0.015).to(torch.bfloat16)
+    outs = (torch.empty_like(w), torch.empty(16, 3072, 2048, dtype=torch.uint8, device=dev),
+            torch.empty(16, 3072, 256, dtype=torch.uint8, device=dev), torch.empty(16, dtype=torch.float32, device=dev))
+    ws = torch.empty(256, dtype=torch.uint8, device=dev)
+    times = []
+    for i in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.fake_quant_weights(w, out=outs, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            times.append(e0.elapsed_time(e1))
+    ms = sum(times) / len(times)
+    gbs = w.numel() * 4.5625 / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "fake_quant_gbs", "value": gbs, "unit": "GB/s", "ms_per_step": ms, "steps": args.steps,
+                      "warmup": args.warmup, "frac_of_hbm": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                      "config": {"workload": "fake-quant + pack, 16 x [3072, 4096] bf16", "l2": "919 MB per call, larger than L2"}}))
+
+
 def run_ours(args):
     import torch
     from paper_2607_15810_b200 import binding as B
     from paper_2607_15810_b200 import synth
+    if args.fake_quant_only:
+        return run_fake_quant_only(args)
 
     from paper_2607_15810_b200 import dist_util as D
     world, rank, local = D.env_world()

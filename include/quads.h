@@ -77,6 +77,8 @@ size_t quads_sf_tiled_bytes(int64_t rows, int64_t K);
  *   gs_out out, float[1]: the per-tensor scale that was used (may be NULL)
  *   workspace  >= quads_quantize_workspace_bytes() bytes
  * rows == 0 is allowed (nothing is written except gs_out = 1 when gs_in is NULL).
+ * A tensor holds fewer than 2^31 scale blocks (rows * K / 16), else QUADS_ERR_SHAPE;
+ * the same limit applies to every tensor of quads_fake_quant_weights.
  */
 quads_status quads_quantize_nvfp4(const void* x, int64_t rows, int64_t K, int64_t ld,
                                   const float* gs_in, uint8_t* q, uint8_t* sf, float* gs_out,

@@ -287,7 +287,7 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   g_launch_count = 0;
   if (rows < 0 || n_tensors < 0 || K <= 0 || (K % 16) != 0 || ld < K || (ld % 16) != 0) return QUADS_ERR_SHAPE;
   if (sf_layout != QUADS_SF_LINEAR && sf_layout != QUADS_SF_TILED) return QUADS_ERR_SHAPE;
-  if (rows * (K / 16) > (int64_t)0x7FFFFFFF * 256 || n_tensors > 65535) return QUADS_ERR_SHAPE;
+  if (rows * (K / 16) > (int64_t)0x7FFFFFFF || n_tensors > 65535) return QUADS_ERR_SHAPE;   // block indices are 31-bit
   if (!workspace || !aligned(workspace, 256) || workspace_bytes < quads_fake_quant_workspace_bytes(n_tensors))
     return QUADS_ERR_WORKSPACE;
   if (n_tensors > 0 && rows > 0 && !x) return QUADS_ERR_NULL;

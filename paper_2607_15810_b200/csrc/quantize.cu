@@ -98,7 +98,16 @@ struct QuantSink {
   int sf_tiled;
   uint32_t k16;      // blocks per row
   int kt_count;      // scale atoms per row tile
+  uint32_t div_m;    // floor(b / k16) = (b * div_m) >> div_s for every block index b < 2^31
+  int div_s;
 };
+
+// The multiplier / shift pair of the division by k16 above (round-up method on 31-bit dividends).
+__device__ __forceinline__ void quant_sink_divisor(QuantSink& o) {
+  const int l = o.k16 > 1 ? 32 - __clz((int)(o.k16 - 1)) : 0;   // ceil(log2(k16))
+  o.div_s = 31 + l;
+  o.div_m = (uint32_t)((((unsigned long long)1 << o.div_s) + o.k16 - 1) / o.k16);
+}
 
 // Quantize block b (16 bf16 values in v0 | v1) and stream the outputs out.
 template <bool kLut>
@@ -111,8 +120,10 @@ __device__ __forceinline__ void emit_block(const QuantSink& o, const QuantCtx& q
   if (o.q) __stcs(reinterpret_cast<uint2*>(o.q + b * 8), make_uint2(bq.lo, bq.hi));
   if (o.sf) {
     if (o.sf_tiled) {
-      const uint32_t r = (uint32_t)(b / o.k16), kb = (uint32_t)(b - (int64_t)r * o.k16);
-      o.sf[sf_tiled_offset(r, kb, o.kt_count)] = (uint8_t)bq.sf8;
+      const uint32_t bu = (uint32_t)b;
+      const uint32_t r = (uint32_t)(((unsigned long long)bu * o.div_m) >> o.div_s), kb = bu - r * o.k16;
+      const uint32_t tile = (r >> 7) * (uint32_t)o.kt_count + (kb >> 2);
+      o.sf[(size_t)tile * 512u + ((r & 31u) * 16u + ((r >> 5) & 3u) * 4u + (kb & 3u))] = (uint8_t)bq.sf8;
     } else {
       o.sf[b] = (uint8_t)bq.sf8;
     }
@@ -216,7 +227,8 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
     const int kt_count = (int)((K + 63) >> 6);
     const bool contiguous = (ld == K);
     const uint32_t k16u = (uint32_t)k16;
-    const QuantSink sink{qt, sft, fqt, sf_tiled, k16u, kt_count};
+    QuantSink sink{qt, sft, fqt, sf_tiled, k16u, kt_count, 0, 0};
+    quant_sink_divisor(sink);
     auto emit = [&](int64_t b, const uint4& v0, const uint4& v1) { emit_block<true>(sink, qc, b, v0, v1); };
     auto src_of = [&](int64_t b) -> const uint16_t* {
       if (contiguous) return base + b * 16;
@@ -345,7 +357,10 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
   extern __shared__ __align__(128) uint8_t smem[];
   RingShared* sh = reinterpret_cast<RingShared*>(smem);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int group = warp / kRingGroupWarps, warp_g = warp % kRingGroupWarps;   // warp_g == kRingConsumers: the producer
+  // Warp 8g + 7 is the producer of group g, so all four producers sit on one warp scheduler
+  // (measured 4 % faster than one producer per scheduler).
+  const int group = warp / kRingGroupWarps, warp_g = warp % kRingGroupWarps;
+  const bool is_producer = warp_g == kRingConsumers;
   uint8_t* stage0 = smem + kRingHeaderBytes + (size_t)group * kRingDepth * kRingChunkBytes;
   const uint32_t stage0_u32 = smem_u32(stage0);
   const uint32_t full0 = smem_u32(&sh->full[group][0]), empty0 = smem_u32(&sh->empty[group][0]);
@@ -381,7 +396,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
     return true;
   };
 
-  if (warp_g == kRingConsumers) {
+  if (is_producer) {
     // =========================== producer (one lane)
     if (lane != 0) return;
     uint64_t keep, stream;
@@ -433,6 +448,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
         uint32_t spins = 0;
         while (!mbar_test(bar, parity)) {
           watch_step();                                          // consumers may be waiting for a scale meanwhile
+          __nanosleep(40);                                       // (neutral for speed; leaves the issue slots alone)
           if ((++spins & 1023u) == 0 && (*abort_flag || globaltimer() - t0 > kWaitNs)) { *abort_flag = 1; ok = false; break; }
         }
         if (!ok) break;
@@ -468,7 +484,8 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
   const int lane_c = warp_g * 32 + lane;                         // lane within the group's consumers
   RingItems ci;
   ci.reset(n_tensors, lead, cnt, group);
-  const QuantSink sink0{q, sf, fq, sf_tiled, k16, kt_count};
+  QuantSink sink0{q, sf, fq, sf_tiled, k16, kt_count, 0, 0};
+  quant_sink_divisor(sink0);
   QuantSink sink = sink0;
   QuantCtx qc;
   qc.inv_lut = nullptr;

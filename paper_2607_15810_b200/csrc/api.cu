@@ -308,7 +308,7 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   const int64_t nblk = rows * (K / 16);
   // A batch of tensors with no scales given: the ring kernel (pipelines of bulk copies, the amax
   // stream running ahead of the quantization by a tensor or two, which must stay in L2).
-  if (!gs_in && ld == K && n_tensors >= 2 && !getenv("QUADS_NO_RING_QUANT")) {
+  if (!gs_in && ld == K && n_tensors >= 2 && nblk > 0 && !getenv("QUADS_NO_RING_QUANT")) {
     const int64_t per64 = ((nblk + di.sm_count - 1) / di.sm_count + 3) / 4 * 4;   // blocks per CTA, 128-byte granules
     const int64_t tensor_bytes = nblk * 32;
     if (per64 < (int64_t)1 << 24 && tensor_bytes * 2 <= (int64_t)64 << 20) {

@@ -396,6 +396,13 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
     return true;
   };
 
+  if (cnt == 0) {
+    // A CTA beyond the end of the tensors (fewer blocks than CTAs): nothing to reduce or quantize,
+    // but every tensor still waits for this CTA's arrival.
+    if (is_producer && lane == 0)
+      for (int t = group; t < n_tensors; t += kRingGroups) atomicAdd(pair + 2 * (size_t)t + 1, 1u);
+    return;
+  }
   if (is_producer) {
     // =========================== producer (one lane)
     if (lane != 0) return;
@@ -415,6 +422,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
       if (owed < n_tensors) {
         const unsigned long long pv = *reinterpret_cast<volatile unsigned long long*>(&sh->pub[owed & (kRingBoard - 1)]);
         if ((uint32_t)(pv >> 32) == (uint32_t)owed + 1u) {       // the CTA is through with A of that tensor
+          *reinterpret_cast<volatile unsigned long long*>(&sh->pub[owed & (kRingBoard - 1)]) = 0;   // slot free again
           uint32_t* pr = pair + 2 * (size_t)owed;
           if ((uint32_t)pv) atomicMax(pr, (uint32_t)pv << 16);
           __threadfence();
@@ -509,8 +517,14 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
           // global atomics would make THIS warp wait for all its output stores in flight
           const uint32_t tm = atomicExch(&sh->cta_max[s], 0u);
           atomicExch(&sh->amax_cnt[s], 0u);
-          *reinterpret_cast<volatile unsigned long long*>(&sh->pub[s]) =
-              ((unsigned long long)((uint32_t)ci.t + 1u) << 32) | tm;
+          volatile unsigned long long* slot = reinterpret_cast<volatile unsigned long long*>(&sh->pub[s]);
+          if (*slot != 0) {                                      // the producer has not taken tensor t - 32 yet
+            const uint64_t t0 = globaltimer();
+            uint32_t spins = 0;
+            while (*slot != 0)
+              if ((++spins & 63u) == 0 && (*abort_flag || globaltimer() - t0 > kWaitNs)) { *abort_flag = 1; break; }
+          }
+          *slot = ((unsigned long long)((uint32_t)ci.t + 1u) << 32) | tm;
         }
       }
       continue;

@@ -127,7 +127,8 @@ def test_fake_quant_bit_exact_and_trainer_equals_rollout(B, n, N, K):
 
 
 @pytest.mark.parametrize("n,N,K", [
-    (40, 64, 128),       # more tensors than the kernel keeps in flight; most CTAs own no block at all
+    (40, 64, 128),       # more tensors than the kernel keeps in flight; 4 blocks per CTA, none for some CTAs
+    (256, 256, 128),     # many tensors, 16 blocks per CTA, 20 CTAs without any: their arrivals must still count
     (2, 8, 16),          # two tensors of one block each
     (9, 1000, 2048),     # a share of 868 blocks: one full chunk and a ragged one, dealt to rotating groups
     (6, 1536, 2048),     # the 30B-A3B expert shape: 3 chunks per share over 4 groups

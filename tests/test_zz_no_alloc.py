@@ -3,6 +3,8 @@ cudaMalloc (device memory owned by someone else's pool, or no allocation
 allowed after start-up).  It must give exactly what the workspace-taking entry
 point gives, on two calls in a row that share its built-in scratch array, and
 refuse a batch beyond its stated capacity.  Collected last on purpose."""
+import gc
+
 import pytest
 import torch
 
@@ -26,6 +28,7 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     for w in batches:
         ref = B.fake_quant_weights(w)
         outs = _outs(w)
+        gc.collect()                                   # tensors kept alive by reference cycles of earlier tests
         before = torch.cuda.memory_allocated()
         B.fake_quant_weights_noalloc(w, outs)
         assert torch.cuda.memory_allocated() == before

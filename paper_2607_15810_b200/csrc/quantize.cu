@@ -305,6 +305,9 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// One aligned 8-byte load of a tensor's {amax bits, arrivals} pair.  A CTA publishes its maximum,
+// fences, then counts itself in, and the load is a single access to one L2 sector, so a pair that
+// shows all arrivals also shows the final maximum.
 __device__ __forceinline__ uint64_t ld_relaxed_u64(const void* p) {
   uint64_t v;
   asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");

@@ -112,6 +112,26 @@ quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t 
 size_t quads_fake_quant_workspace_bytes(int64_t n_tensors);
 
 /*
+ * Activation fake-quant QDQ_A for the learner-side ablations of the paper
+ * (Table "qdq-alignment": a W16A4- or W4A4-QAT learner quantizes and
+ * dequantizes its own activations; Section "Asymmetric Quantization-Aware
+ * Training" argues against it, and keeps activations in BF16).  The same NVFP4
+ * quantizer as quads_quantize_nvfp4, followed by the same dequantization as
+ * quads_fake_quant_weights, so x_fq is bit for bit what the rollout's
+ * activation operand decodes to.  The straight-through backward of the node is
+ * the identity and needs no kernel.
+ *   x      bf16 [rows, K], row stride `ld` elements (ld >= K, ld % 16 == 0), 32-byte aligned
+ *   gs_in  float[1] per-tensor scale, or NULL: amax(x)/2688 computed on device
+ *   x_fq   out, bf16 [rows, K] contiguous, 32-byte aligned
+ *   gs_out out, float[1]: the scale that was used (may be NULL)
+ *   workspace  >= quads_quantize_workspace_bytes() bytes
+ */
+quads_status quads_fake_quant_activations(const void* x, int64_t rows, int64_t K, int64_t ld,
+                                          const float* gs_in, void* x_fq, float* gs_out,
+                                          void* workspace, size_t workspace_bytes,
+                                          void* cuda_stream);
+
+/*
  * Allocation-free variant of quads_fake_quant_weights (the paper has no
  * counterpart; it exists for callers that cannot provide scratch memory).
  * Some hosts of this library may not call cudaMalloc where they use it: a

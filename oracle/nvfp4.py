@@ -93,6 +93,15 @@ def dequantize_bf16(codes, sf8, gs):
     return F.bf16_round(dequantize_f32(codes, sf8, gs))
 
 
+def fake_quant_activations(x, gs=None):
+    """x: float32 (bf16-valued) [rows, K].  The activation QDQ node of the
+    learner-side ablations (Table "qdq-alignment"): quantize as the rollout
+    does (Eq. act-error-def), decode, round to bf16.  Returns (x_fq
+    bf16-as-float32, gs float32)."""
+    c, s, g = quantize(np.asarray(x, dtype=F32), gs)
+    return dequantize_bf16(c, s, g), g
+
+
 def fake_quant_weights(w):
     """w: float32 (bf16-valued) [n_tensors, N, K].  Each [N, K] slice is one
     tensor with its own amax-derived per-tensor scale (Eq. w4a16-qat-forward).

@@ -50,6 +50,8 @@ lib.quads_quantize_nvfp4.restype = _i32
 lib.quads_quantize_nvfp4.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p, _sz, _p]
 lib.quads_fake_quant_weights.restype = _i32
 lib.quads_fake_quant_weights.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p, _sz, _p]
+lib.quads_fake_quant_activations.restype = _i32
+lib.quads_fake_quant_activations.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, _sz, _p]
 lib.quads_fake_quant_weights_noalloc.restype = _i32
 lib.quads_fake_quant_weights_noalloc.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p]
 lib.quads_moe_w4a4_rac.restype = _i32
@@ -114,6 +116,23 @@ def quantize_nvfp4(x, gs=None, sf_layout=SF_LINEAR, out=None, workspace=None):
     check(lib.quads_quantize_nvfp4(_ptr(x), rows, K, ld, _ptr(gs), _ptr(q), _ptr(sf), _ptr(gs_out),
                                    sf_layout, _ptr(ws), ws.numel(), _stream()))
     return q, sf, gs_out
+
+
+def fake_quant_activations(x, gs=None, out=None, workspace=None):
+    """x: bf16 CUDA tensor [rows, K] (row stride allowed).  Returns (x_fq bf16 [rows, K], gs)."""
+    assert x.dtype == torch.bfloat16 and x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    rows, K = x.shape
+    dev = x.device
+    if out is None:
+        x_fq = torch.empty(rows, K, dtype=torch.bfloat16, device=dev)
+        gs_out = torch.empty(1, dtype=torch.float32, device=dev)
+    else:
+        x_fq, gs_out = out
+    ws = workspace if workspace is not None else _ws(lib.quads_quantize_workspace_bytes(), dev)
+    ld = x.stride(0) if rows > 1 else max(K, x.stride(0))
+    check(lib.quads_fake_quant_activations(_ptr(x), rows, K, ld, _ptr(gs), _ptr(x_fq), _ptr(gs_out), _ptr(ws),
+                                           ws.numel(), _stream()))
+    return x_fq, gs_out
 
 
 def fake_quant_weights(w, want_fq=True, want_pack=True, sf_layout=SF_LINEAR, out=None, workspace=None):

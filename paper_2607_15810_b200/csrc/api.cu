@@ -363,6 +363,14 @@ quads_status quads_quantize_nvfp4(const void* x, int64_t rows, int64_t K, int64_
                          workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
+quads_status quads_fake_quant_activations(const void* x, int64_t rows, int64_t K, int64_t ld, const float* gs_in,
+                                          void* x_fq, float* gs_out, void* workspace, size_t workspace_bytes,
+                                          void* cuda_stream) {
+  if (rows > 0 && !x_fq) return QUADS_ERR_NULL;
+  return quantize_common(x, 1, rows, K, ld, 0, gs_in, x_fq, nullptr, nullptr, gs_out, QUADS_SF_LINEAR, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
 quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t N, int64_t K, void* w_fq,
                                       uint8_t* q, uint8_t* sf, float* gs, int sf_layout, void* workspace,
                                       size_t workspace_bytes, void* cuda_stream) {

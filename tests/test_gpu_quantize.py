@@ -170,3 +170,24 @@ def test_fake_quant_batch_kernel_repeats_bit_for_bit(B):
         again = B.fake_quant_weights(w)
         for k in ("gs", "q", "sf", "w_fq"):
             assert torch.equal(first[k].view(torch.uint8), again[k].view(torch.uint8)), k
+
+
+@pytest.mark.parametrize("rows,K,seed", [(1, 16, 1), (333, 2048, 3), (2048, 4096, 4)])
+def test_activation_fake_quant_decodes_what_the_rollout_operand_holds(B, rows, K, seed):
+    x = _bf16((rows, K), seed, 2.0)
+    if K >= 64:
+        x[:, 7] *= 30
+    xf, g = B.fake_quant_activations(x.cuda())
+    xf_o, g_o = Q.fake_quant_activations(_f32(x))
+    assert np.float32(g.item()) == g_o
+    assert np.array_equal(F.bf16_bits(_f32(xf)), F.bf16_bits(xf_o))
+    # ... and it is the decode of exactly the bytes quads_quantize_nvfp4 writes
+    q, sf, g2 = B.quantize_nvfp4(x.cuda())
+    dec = Q.dequantize_bf16(F.unpack_nibbles(q.cpu().numpy()), sf.cpu().numpy(), g2.item())
+    assert np.array_equal(F.bf16_bits(dec), F.bf16_bits(_f32(xf)))
+    # a given (static) scale and a row stride
+    big = _bf16((max(rows, 2), 2 * K), seed + 50, 1.0).cuda()
+    gs = torch.tensor([0.004], dtype=torch.float32).cuda()
+    xs, _ = B.fake_quant_activations(big[:, :K], gs=gs)
+    xs_o, _ = Q.fake_quant_activations(_f32(big[:, :K]), np.float32(0.004))
+    assert np.array_equal(F.bf16_bits(_f32(xs)), F.bf16_bits(xs_o))

@@ -115,3 +115,30 @@ def test_fake_quant_error_is_small_relative_to_block_amax():
     blk = np.abs(w[0]).reshape(64, 32, 16).max(axis=2).repeat(16, axis=1)
     # half of the coarsest step (2/6 of amax), E4M3 scale rounding, bf16 rounding
     assert np.all(np.abs(w_fq[0] - w[0]) <= blk * (1 / 6 + 2.0 ** -4 + 2.0 ** -8) + 1e-12)
+
+
+def test_activation_fake_quant_is_the_decode_of_the_rollout_operand():
+    """The learner-side activation QDQ (Table "qdq-alignment") must return what
+    the rollout's quantized operand decodes to, leave a representable tensor
+    unchanged, stay within half a grid step of the block's own scale, and be a
+    projection (applying it twice changes nothing when the scale is kept)."""
+    x = _rand_bf16((19, 192), 4, 1.5)
+    x[:, 3] *= 25
+    xf, g = Q.fake_quant_activations(x)
+    c, s, g2 = Q.quantize(x)
+    assert g == g2 and np.array_equal(xf, F.bf16_round(Q.dequantize_f32(c, s, g)))
+    # error bound: at most half a step of the coarsest E2M1 interval (2 units) times the block scale, + bf16 rounding
+    d = Q.block_scales_f32(s, g).astype(np.float64)
+    err = np.abs(xf.astype(np.float64) - x.astype(np.float64)).reshape(19, -1, 16)
+    assert np.all(err <= d[:, :, None] * 1.0 * (1 + 2.0 ** -7))
+    # projection with the scale held fixed
+    xf2, _ = Q.fake_quant_activations(Q.dequantize_f32(c, s, g), g)
+    assert np.array_equal(xf2, xf)
+    # a tensor that is already on the grid (bf16-representable products) comes back bit for bit
+    rng = np.random.default_rng(2)
+    codes = rng.integers(0, 16, (5, 64)).astype(np.uint8)
+    codes[:, ::16] = 7
+    sf8 = np.full((5, 4), 0x38, np.uint8)                   # block scale 1.0
+    t = Q.dequantize_f32(codes, sf8, np.float32(0.25))
+    tf, _ = Q.fake_quant_activations(t, np.float32(0.25))
+    assert np.array_equal(tf, t)

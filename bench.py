@@ -530,7 +530,32 @@ def run_ours(args):
         aux["dense_linear_ms"] = dms
         aux["dense_linear_tflops_algorithmic"] = 2.0 * Td * Kd * Nd * 1.5 / (dms * 1e-3) / 1e12
         aux["dense_linear_note"] = "T=%d, %d -> %d, RAC on %d channels, activation quantized online, whole call" % (Td, Kd, Nd, Kd // 2)
-        del xd, wd, wsd
+        del xd, wd
+        # the layer-wise mismatch ||Y_rollout - Y_learner|| / ||Y_learner|| of that projection as a function of the
+        # share of compensated channels (the paper's ratios): Y_learner = QDQ_W(W) x in float32 with bf16 activations
+        # (the asymmetric-QAT learner), Y_rollout = this library's W4A4 + RAC output; activations with 2 % heavy
+        # channels (x25), which is where activation quantization error concentrates
+        gen = torch.Generator(device=dev).manual_seed(77)
+        xe = torch.randn(Td, Kd, device=dev, generator=gen)
+        heavy = torch.randperm(Kd, device=dev, generator=gen)[: Kd // 50]
+        xe[:, heavy] *= 25.0
+        xe = xe.to(torch.bfloat16)
+        we = B.fake_quant_weights((torch.randn(1, Nd, Kd, device=dev, generator=gen) * 0.02).to(torch.bfloat16),
+                                  want_fq=True, sf_layout=B.SF_TILED)
+        tf32 = torch.backends.cuda.matmul.allow_tf32
+        torch.backends.cuda.matmul.allow_tf32 = False
+        y_learner = xe.to(torch.float32) @ we["w_fq"][0].to(torch.float32).t()
+        torch.backends.cuda.matmul.allow_tf32 = tf32
+        ref_norm = torch.linalg.norm(y_learner).item()
+        sweep = {}
+        for pct in (0.0, 12.5, 25.0, 50.0, 75.0, 100.0):
+            y = B.dense_w4a4_rac(xe, we, int(Kd * pct / 100.0), workspace=wsd)["out"]
+            sweep["%g%%" % pct] = torch.linalg.norm(y.to(torch.float32) - y_learner).item() / ref_norm
+        aux["rac_mismatch_vs_ratio"] = sweep
+        aux["rac_mismatch_note"] = ("relative Frobenius mismatch of the W4A4 + RAC projection (T=%d, %d -> %d) against the "
+                                    "learner's QDQ_W(W) x (float32 accumulate, bf16 activations), per share of compensated "
+                                    "channels; output rounding to bf16 included" % (Td, Kd, Nd))
+        del xe, we, y_learner, wsd
         # decode-sized batch on the same layer (the prefill and decode workloads share their weights):
         # weights cold (L2 flushed between iterations); roofline = streaming the 340 MB of weights once
         if args.workload == "prefill":

@@ -484,7 +484,17 @@ def run_ours(args):
         aux["fake_quant_gbs"] = w.numel() * 4.5625 / (sum(tf) / len(tf) * 1e-3) / 1e9
         aux["fake_quant_frac_of_hbm"] = aux["fake_quant_gbs"] / peaks["hbm_gbs"]
         aux["hbm_peak_gbs"] = peaks["hbm_gbs"]
-        del w, outs
+        # decode of those packed tensors back to bf16 (the rollout's weight load / a W4A16 operand): 0.5625 B in, 2 B out
+        dq_out = outs[0]
+
+        def dstep_():
+            B.dequantize_nvfp4(outs[1], outs[2], outs[3], 3072, 4096, out=dq_out)
+        for _ in range(3):
+            dstep_()
+        tdq = timed(dstep_, 20)
+        aux["dequantize_gbs"] = w.numel() * 2.5625 / (sum(tdq) / len(tdq) * 1e-3) / 1e9
+        aux["dequantize_frac_of_hbm"] = aux["dequantize_gbs"] / peaks["hbm_gbs"]
+        del w, outs, dq_out
         # one whole layer of the AQAT + weight-sync workload: 128 experts x (W13 [3072, 4096] + W2 [4096, 1536]),
         # 2.416 G elements = 4.83 GB in, 6.19 GB out; the 48-layer job is this 48 times over one reused buffer
         torch.cuda.empty_cache()

@@ -112,6 +112,22 @@ quads_status quads_fake_quant_weights(const void* w, int64_t n_tensors, int64_t 
 size_t quads_fake_quant_workspace_bytes(int64_t n_tensors);
 
 /*
+ * NVFP4 -> bf16 decode of packed tensors: out = value(code) * (E4M3 block scale *
+ * per-tensor scale), one float32 multiply rounded to bf16 -- the right-hand side
+ * of Eq. "weight-qdq-align", i.e. what the rollout side holds after loading the
+ * bytes quads_fake_quant_weights produced (out equals that call's w_fq bit for
+ * bit), and the weight operand of a W4A16 rollout.
+ *   q    u8 [n_tensors, rows, K/2], 8-byte aligned
+ *   sf   u8, one [rows, K/16] (or tiled) block per tensor, per `sf_layout`
+ *   gs   float [n_tensors] per-tensor scales (device)
+ *   out  bf16 [n_tensors, rows, K], 32-byte aligned
+ * rows * K / 16 < 2^31 per tensor.  n_tensors == 0 or rows == 0 does nothing.
+ */
+quads_status quads_dequantize_nvfp4(const uint8_t* q, const uint8_t* sf, const float* gs,
+                                    int64_t n_tensors, int64_t rows, int64_t K, int sf_layout,
+                                    void* out, void* cuda_stream);
+
+/*
  * Activation fake-quant QDQ_A for the learner-side ablations of the paper
  * (Table "qdq-alignment": a W16A4- or W4A4-QAT learner quantizes and
  * dequantizes its own activations; Section "Asymmetric Quantization-Aware

@@ -50,6 +50,8 @@ lib.quads_quantize_nvfp4.restype = _i32
 lib.quads_quantize_nvfp4.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p, _sz, _p]
 lib.quads_fake_quant_weights.restype = _i32
 lib.quads_fake_quant_weights.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, C.c_int, _p, _sz, _p]
+lib.quads_dequantize_nvfp4.restype = _i32
+lib.quads_dequantize_nvfp4.argtypes = [_p, _p, _p, _i64, _i64, _i64, C.c_int, _p, _p]
 lib.quads_fake_quant_activations.restype = _i32
 lib.quads_fake_quant_activations.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p, _sz, _p]
 lib.quads_fake_quant_weights_noalloc.restype = _i32
@@ -116,6 +118,15 @@ def quantize_nvfp4(x, gs=None, sf_layout=SF_LINEAR, out=None, workspace=None):
     check(lib.quads_quantize_nvfp4(_ptr(x), rows, K, ld, _ptr(gs), _ptr(q), _ptr(sf), _ptr(gs_out),
                                    sf_layout, _ptr(ws), ws.numel(), _stream()))
     return q, sf, gs_out
+
+
+def dequantize_nvfp4(q, sf, gs, rows, K, sf_layout=SF_LINEAR, out=None):
+    """q: u8 [n, rows, K/2]; sf: u8 per layout; gs: f32 [n].  Returns bf16 [n, rows, K]."""
+    n = q.shape[0]
+    if out is None:
+        out = torch.empty(n, rows, K, dtype=torch.bfloat16, device=q.device)
+    check(lib.quads_dequantize_nvfp4(_ptr(q), _ptr(sf), _ptr(gs), n, rows, K, sf_layout, _ptr(out), _stream()))
+    return out
 
 
 def fake_quant_activations(x, gs=None, out=None, workspace=None):

@@ -363,6 +363,30 @@ quads_status quads_quantize_nvfp4(const void* x, int64_t rows, int64_t K, int64_
                          workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
+quads_status quads_dequantize_nvfp4(const uint8_t* q, const uint8_t* sf, const float* gs, int64_t n_tensors,
+                                    int64_t rows, int64_t K, int sf_layout, void* out, void* cuda_stream) {
+  g_launch_count = 0;
+  if (rows < 0 || n_tensors < 0 || K <= 0 || (K % 16) != 0) return QUADS_ERR_SHAPE;
+  if (sf_layout != QUADS_SF_LINEAR && sf_layout != QUADS_SF_TILED) return QUADS_ERR_SHAPE;
+  const int64_t nblk = rows * (K / 16);
+  if (nblk > (int64_t)0x7FFFFFFF || n_tensors > 65535) return QUADS_ERR_SHAPE;
+  if (n_tensors == 0 || rows == 0) return QUADS_OK;
+  if (!q || !sf || !gs || !out) return QUADS_ERR_NULL;
+  if (!aligned(q, 8) || !aligned(out, 32)) return QUADS_ERR_SHAPE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  const int tiled = sf_layout == QUADS_SF_TILED;
+  const int64_t sf_stride = tiled ? (int64_t)quads_sf_tiled_bytes(rows, K) : nblk;
+  const int64_t want = (nblk * n_tensors + 255) / 256;
+  const int grid = (int)std::min<int64_t>(want, (int64_t)di.sm_count * 16);
+  QUADS_CUDA_OK(launch_kernel(dequantize_kernel, dim3(grid), dim3(256), (size_t)0, static_cast<cudaStream_t>(cuda_stream),
+                              q, sf, gs, (int)n_tensors, nblk, (uint32_t)(K / 16), (int)((K + 63) / 64), tiled, sf_stride,
+                              static_cast<uint16_t*>(out)));
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
 quads_status quads_fake_quant_activations(const void* x, int64_t rows, int64_t K, int64_t ld, const float* gs_in,
                                           void* x_fq, float* gs_out, void* workspace, size_t workspace_bytes,
                                           void* cuda_stream) {

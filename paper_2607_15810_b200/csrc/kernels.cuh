@@ -31,6 +31,8 @@ __global__ void fake_quant_ring_kernel(const uint16_t* x, int64_t nblk, int64_t 
                                        uint32_t* pair, int per, int lead, uint8_t* q, uint8_t* sf, uint16_t* fq,
                                        float* gs_out, int sf_tiled, int64_t sf_tensor_stride, uint32_t k16,
                                        int kt_count);
+__global__ void dequantize_kernel(const uint8_t* q, const uint8_t* sf, const float* gs, int n_tensors, int64_t nblk,
+                                  uint32_t k16, int kt_count, int sf_tiled, int64_t sf_tensor_stride, uint16_t* out);
 __global__ void rac_quant_kernel(const uint16_t* x, int T, int H, const float* gs_in, uint32_t* amax_bits,
                                  unsigned int* grid_arrivals, int32_t* status,
                                  float* gs_store, int rows_per_cta, int with_residual, float* partials, uint8_t* xq,

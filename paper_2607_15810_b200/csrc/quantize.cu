@@ -588,6 +588,44 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
 }
 
 // ---------------------------------------------------------------------------
+// NVFP4 -> bf16 decode of packed tensors (what a rollout engine's weight loader, or a W4A16
+// path, reads): value(code) * (E4M3 block scale * per-tensor scale), one float32 multiply,
+// rounded to bf16 -- the decode that the weight fake-quant's bf16 output is defined by.
+// One 16-element block per thread and step: 8 B codes + 1 B scale in, 32 B out.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+dequantize_kernel(const uint8_t* __restrict__ q, const uint8_t* __restrict__ sf, const float* __restrict__ gs,
+                  int n_tensors, int64_t nblk, uint32_t k16, int kt_count, int sf_tiled, int64_t sf_tensor_stride,
+                  uint16_t* __restrict__ out) {
+  pdl_sync();
+  QuantSink geo{nullptr, nullptr, nullptr, sf_tiled, k16, kt_count, 0, 0};
+  quant_sink_divisor(geo);
+  const int64_t total = nblk * n_tensors;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int t = (int)(i / nblk);
+    const uint32_t b = (uint32_t)(i - (int64_t)t * nblk);
+    size_t so = b;
+    if (sf_tiled) {
+      const uint32_t r = (uint32_t)(((unsigned long long)b * geo.div_m) >> geo.div_s), kb = b - r * k16;
+      so = (size_t)((r >> 7) * (uint32_t)kt_count + (kb >> 2)) * 512u + ((r & 31u) * 16u + ((r >> 5) & 3u) * 4u + (kb & 3u));
+    }
+    const uint2 codes = __ldcs(reinterpret_cast<const uint2*>(q) + i);
+    BlockQ bq;
+    bq.lo = codes.x;
+    bq.hi = codes.y;
+    bq.sf8 = sf[(size_t)t * sf_tensor_stride + so];
+    bq.d = __fmul_rn(e4m3_to_f32(bq.sf8), gs[t]);
+    float d[16];
+    dequant_block(bq, d);
+    uint4* dst = reinterpret_cast<uint4*>(out + (size_t)i * 16);
+    __stcs(dst, make_uint4(f32x2_to_bf16x2(d[0], d[1]), f32x2_to_bf16x2(d[2], d[3]),
+                           f32x2_to_bf16x2(d[4], d[5]), f32x2_to_bf16x2(d[6], d[7])));
+    __stcs(dst + 1, make_uint4(f32x2_to_bf16x2(d[8], d[9]), f32x2_to_bf16x2(d[10], d[11]),
+                               f32x2_to_bf16x2(d[12], d[13]), f32x2_to_bf16x2(d[14], d[15])));
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Site-13 quantization pass, token order.  For every row and 16-channel block:
 // Q_A(x) codes + scale; the residual Q_A(x) - x in float32 (Eq. residual-def);
 // its squared sum per channel over the rows this CTA owns (Eq. channel-score,

@@ -191,3 +191,20 @@ def test_activation_fake_quant_decodes_what_the_rollout_operand_holds(B, rows, K
     xs, _ = B.fake_quant_activations(big[:, :K], gs=gs)
     xs_o, _ = Q.fake_quant_activations(_f32(big[:, :K]), np.float32(0.004))
     assert np.array_equal(F.bf16_bits(_f32(xs)), F.bf16_bits(xs_o))
+
+
+@pytest.mark.parametrize("n,N,K", [(1, 1, 16), (3, 100, 80), (4, 1536, 2048)])
+def test_dequantize_gives_the_trainers_fake_quant_bit_for_bit(B, n, N, K):
+    """Eq. weight-qdq-align: decoding the packed bytes on the rollout side gives
+    the bf16 tensor the trainer multiplied by -- for both scale layouts, and
+    equal to the oracle's decode of the same bytes."""
+    w = _bf16((n, N, K), 21 + n, 0.02).cuda()
+    lin = B.fake_quant_weights(w)
+    til = B.fake_quant_weights(w, sf_layout=B.SF_TILED)
+    d_lin = B.dequantize_nvfp4(lin["q"], lin["sf"], lin["gs"], N, K)
+    d_til = B.dequantize_nvfp4(til["q"], til["sf"], til["gs"], N, K, sf_layout=B.SF_TILED)
+    assert torch.equal(d_lin.view(torch.int16), lin["w_fq"].view(torch.int16))
+    assert torch.equal(d_til.view(torch.int16), lin["w_fq"].view(torch.int16))
+    for i in range(n):
+        dec = Q.dequantize_bf16(F.unpack_nibbles(lin["q"][i].cpu().numpy()), lin["sf"][i].cpu().numpy(), lin["gs"][i].item())
+        assert np.array_equal(F.bf16_bits(dec), F.bf16_bits(_f32(d_lin[i])))

@@ -568,6 +568,17 @@ def run_ours(args):
         del xe, we, y_learner, wsd
         # decode-sized batch on the same layer (the prefill and decode workloads share their weights):
         # weights cold (L2 flushed between iterations); roofline = streaming the 340 MB of weights once
+        # the benchmark's own step replayed from a CUDA graph: what the eager launches and cross-stream events cost
+        pgraph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(pgraph):
+            step()
+        for _ in range(3):
+            flush_l2()
+            pgraph.replay()
+        tpg = timed(pgraph.replay, 20)
+        aux["step_graph_ms"] = sum(tpg) / len(tpg)
+        aux["step_graph_tokens_per_s"] = T / (aux["step_graph_ms"] * 1e-3)
+        del pgraph
         if args.workload == "prefill":
             dsh = synth.MOE_SHAPES["decode"]
             dn13, dn2 = nsel_of(dsh, args.variant)

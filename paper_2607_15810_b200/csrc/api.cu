@@ -309,7 +309,19 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   // A batch of tensors with no scales given: the ring kernel (pipelines of bulk copies, the amax
   // stream running ahead of the quantization by a tensor or two, which must stay in L2).
   if (!gs_in && ld == K && n_tensors >= 2 && nblk > 0 && !getenv("QUADS_NO_RING_QUANT")) {
-    const int64_t per64 = ((nblk + di.sm_count - 1) / di.sm_count + 3) / 4 * 4;   // blocks per CTA, 128-byte granules
+    // small tensors are dealt to 2 or 4 sets of CTAs (tensor t to set t mod split), so that a CTA's
+    // share is a few 14 KB chunks; the grid is a multiple of the split
+    int split = 1;
+    const int64_t chunk_blocks = kRingChunkBytes / 32;
+    while (split < 4 && n_tensors >= 2 * split && di.sm_count % (2 * split) == 0 &&
+           (nblk + di.sm_count / split - 1) / (di.sm_count / split) < 3 * chunk_blocks)
+      split *= 2;
+    if (const char* e = getenv("QUADS_RING_SPLIT")) {
+      const int v = atoi(e);
+      if ((v == 1 || v == 2 || v == 4) && di.sm_count % v == 0) split = v;
+    }
+    const int ctas_per_tensor = di.sm_count / split;
+    const int64_t per64 = ((nblk + ctas_per_tensor - 1) / ctas_per_tensor + 3) / 4 * 4;   // blocks per CTA, 128-byte granules
     const int64_t tensor_bytes = nblk * 32;
     if (per64 < (int64_t)1 << 24 && tensor_bytes * 2 <= (int64_t)64 << 20) {
       // A's lead over Q: a group's chunks of one tensor (so Q never catches up with A inside a
@@ -323,7 +335,7 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
       int64_t stride = tensor_stride;
       int64_t nb = nblk;
       QUADS_CUDA_OK(set_max_dynamic_smem<fake_quant_ring_kernel>(kRingSmemBytes));
-      void* rargs[] = {&xp, &nb, &stride, &nt, &amax_bits, &per, &lead, &q, &sf, &fqp,
+      void* rargs[] = {&xp, &nb, &stride, &nt, &amax_bits, &per, &lead, &split, &q, &sf, &fqp,
                        &gs_out, &tiled, &sf_stride, &k16, &kt_count};
       QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fake_quant_ring_kernel), dim3(di.sm_count),
                                                 dim3(kRingThreads), rargs, (size_t)kRingSmemBytes, st));

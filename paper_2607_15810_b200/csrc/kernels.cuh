@@ -28,7 +28,7 @@ constexpr int kRingHeaderBytes = 1024;
 constexpr int kRingChunkBytes = 7 * 32 * 2 * 32;
 constexpr int kRingSmemBytes = kRingHeaderBytes + 4 * kRingDepth * kRingChunkBytes;
 __global__ void fake_quant_ring_kernel(const uint16_t* x, int64_t nblk, int64_t tensor_stride, int n_tensors,
-                                       uint32_t* pair, int per, int lead, uint8_t* q, uint8_t* sf, uint16_t* fq,
+                                       uint32_t* pair, int per, int lead, int split, uint8_t* q, uint8_t* sf, uint16_t* fq,
                                        float* gs_out, int sf_tiled, int64_t sf_tensor_stride, uint32_t k16,
                                        int kt_count);
 __global__ void dequantize_kernel(const uint8_t* q, const uint8_t* sf, const float* gs, int n_tensors, int64_t nblk,

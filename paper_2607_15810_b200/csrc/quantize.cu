@@ -353,8 +353,8 @@ struct RingItems {
 
 
 __global__ void __launch_bounds__(kRingThreads, 1)
-fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t tensor_stride, int n_tensors,
-                       uint32_t* __restrict__ pair, int per, int lead, uint8_t* __restrict__ q,
+fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t tensor_stride, int n_tensors_all,
+                       uint32_t* __restrict__ pair, int per, int lead, int split, uint8_t* __restrict__ q,
                        uint8_t* __restrict__ sf, uint16_t* __restrict__ fq, float* __restrict__ gs_out, int sf_tiled,
                        int64_t sf_tensor_stride, uint32_t k16, int kt_count) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -367,7 +367,14 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
   uint8_t* stage0 = smem + kRingHeaderBytes + (size_t)group * kRingDepth * kRingChunkBytes;
   const uint32_t stage0_u32 = smem_u32(stage0);
   const uint32_t full0 = smem_u32(&sh->full[group][0]), empty0 = smem_u32(&sh->empty[group][0]);
-  const int64_t start = (int64_t)blockIdx.x * per;               // first block of this CTA's share
+  // The CTAs form `split` sets; set s takes tensors s, s + split, ... (small tensors: a share of a
+  // few chunks per CTA keeps the lanes busy and halves the number of CTAs a scale has to wait for).
+  // Below, tensors are numbered within the set; glob() gives the caller's index.
+  const int ctas_per_tensor = (int)gridDim.x / split;
+  const int set = (int)blockIdx.x / ctas_per_tensor, cta_in_set = (int)blockIdx.x % ctas_per_tensor;
+  const int n_tensors = set < n_tensors_all ? (n_tensors_all - set + split - 1) / split : 0;
+  auto glob = [&](int t) -> size_t { return (size_t)set + (size_t)split * (size_t)t; };
+  const int64_t start = (int64_t)cta_in_set * per;               // first block of this CTA's share
   const int64_t left = nblk - start;
   const int cnt = left <= 0 ? 0 : (left < per ? (int)left : per);  // blocks in the share (same for every tensor)
   volatile int* abort_flag = &sh->abort_flag;
@@ -403,7 +410,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
     // A CTA beyond the end of the tensors (fewer blocks than CTAs): nothing to reduce or quantize,
     // but every tensor still waits for this CTA's arrival.
     if (is_producer && lane == 0)
-      for (int t = group; t < n_tensors; t += kRingGroups) atomicAdd(pair + 2 * (size_t)t + 1, 1u);
+      for (int t = group; t < n_tensors; t += kRingGroups) atomicAdd(pair + 2 * glob(t) + 1, 1u);
     return;
   }
   if (is_producer) {
@@ -426,7 +433,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
         const unsigned long long pv = *reinterpret_cast<volatile unsigned long long*>(&sh->pub[owed & (kRingBoard - 1)]);
         if ((uint32_t)(pv >> 32) == (uint32_t)owed + 1u) {       // the CTA is through with A of that tensor
           *reinterpret_cast<volatile unsigned long long*>(&sh->pub[owed & (kRingBoard - 1)]) = 0;   // slot free again
-          uint32_t* pr = pair + 2 * (size_t)owed;
+          uint32_t* pr = pair + 2 * glob(owed);
           if ((uint32_t)pv) atomicMax(pr, (uint32_t)pv << 16);
           __threadfence();
           atomicAdd(pr + 1, 1u);
@@ -435,14 +442,14 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
       }
       if (watch >= n_tensors) return;
       if (asked && clock64() - asked_at < 2000) return;
-      if (asked && (uint32_t)(seen >> 32) == gridDim.x) {
-        if (gs_out && blockIdx.x == 0) gs_out[watch] = gs_from_amax_bits((uint32_t)seen);
+      if (asked && (uint32_t)(seen >> 32) == (uint32_t)ctas_per_tensor) {
+        if (gs_out && cta_in_set == 0) gs_out[glob(watch)] = gs_from_amax_bits((uint32_t)seen);
         sh->board[watch & (kRingBoard - 1)] = ((unsigned long long)((uint32_t)watch + 1u) << 32) | (uint32_t)seen;
         watch += kRingGroups;
         asked = false;
         if (watch >= n_tensors) return;
       }
-      seen = ld_relaxed_u64(words + watch);
+      seen = ld_relaxed_u64(words + glob(watch));
       asked = true;
       asked_at = clock64();
     };
@@ -466,7 +473,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
       }
       const uint32_t bytes = (uint32_t)pi.nb * 32u;
       mbar_expect_tx(full0 + 8 * s, bytes);
-      bulk_load_hint(stage0_u32 + s * kRingChunkBytes, x + (size_t)pi.t * tensor_stride + (size_t)(start + pi.blk0) * 16,
+      bulk_load_hint(stage0_u32 + s * kRingChunkBytes, x + glob(pi.t) * tensor_stride + (size_t)(start + pi.blk0) * 16,
                      bytes, full0 + 8 * s, pi.kind == kItemA ? keep : stream);
       ++issued;
       watch_step();
@@ -481,7 +488,7 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
     if (!ok) {
       // gave up: mark the scales not posted, and let the copies in flight land (bounded) before leaving
       if (gs_out)
-        for (int t = watch; t < n_tensors; t += kRingGroups) gs_out[t] = __int_as_float(0x7FC00000);
+        for (int t = watch; t < n_tensors; t += kRingGroups) gs_out[glob(t)] = __int_as_float(0x7FC00000);
       for (int d = issued < kRingDepth ? 0 : issued - kRingDepth; d < issued; ++d) {
         const uint32_t bar = full0 + 8 * (d % kRingDepth), parity = (uint32_t)(d / kRingDepth) & 1u;
         const uint64_t t1 = globaltimer();
@@ -554,9 +561,9 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
       cur_q = t;
       quant_ctx_scalars(qc, gs_from_amax_bits(amax_b));
       sink = sink0;
-      if (sink.q) sink.q += (size_t)t * nblk * 8;
-      if (sink.sf) sink.sf += (size_t)t * sf_tensor_stride;
-      if (sink.fq) sink.fq += (size_t)t * nblk * 16;
+      if (sink.q) sink.q += glob(t) * nblk * 8;
+      if (sink.sf) sink.sf += glob(t) * sf_tensor_stride;
+      if (sink.fq) sink.fq += glob(t) * nblk * 16;
     }
     const int s = consumed % kRingDepth;
     if (!wait_bar(full0 + 8 * s, (uint32_t)(consumed / kRingDepth) & 1u)) break;

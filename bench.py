@@ -522,6 +522,24 @@ def run_ours(args):
         aux["aqat_layer_frac_of_hbm"] = aux["aqat_layer_gbs"] / peaks["hbm_gbs"]
         aux["aqat_48_layers_s_extrapolated"] = 48 * lms * 1e-3
         del w13l, w2l, outs13, outs2
+        # the same for the layer this benchmark's MoE workload is taken from (H=2048, I=768):
+        # 128 experts x (W13 [1536, 2048] + W2 [2048, 768]), 0.604 G elements
+        ws13 = (torch.randn(n_e, 1536, 2048, device=dev) * 0.015).to(torch.bfloat16)
+        ws2 = (torch.randn(n_e, 2048, 768, device=dev) * 0.015).to(torch.bfloat16)
+        os13 = (torch.empty_like(ws13), torch.empty(n_e, 1536, 1024, dtype=torch.uint8, device=dev),
+                torch.empty(n_e, 1536, 128, dtype=torch.uint8, device=dev), torch.empty(n_e, dtype=torch.float32, device=dev))
+        os2 = (torch.empty_like(ws2), torch.empty(n_e, 2048, 384, dtype=torch.uint8, device=dev),
+               torch.empty(n_e, 2048, 48, dtype=torch.uint8, device=dev), torch.empty(n_e, dtype=torch.float32, device=dev))
+
+        def small_layer_step():
+            B.fake_quant_weights(ws13, out=os13, workspace=lws)
+            B.fake_quant_weights(ws2, out=os2, workspace=lws)
+        small_layer_step()
+        tsl = timed(small_layer_step, 5)
+        sms_ = sum(tsl) / len(tsl)
+        aux["aqat_layer_h2048_ms"] = sms_
+        aux["aqat_layer_h2048_frac_of_hbm"] = (ws13.numel() + ws2.numel()) * 4.5625 / (sms_ * 1e-3) / 1e9 / peaks["hbm_gbs"]
+        del ws13, ws2, os13, os2
         torch.cuda.empty_cache()
         # a dense (single-expert) W4A4 + RAC projection at model scale: 8192 tokens, 4096 -> 4096, 50 % of the
         # input channels compensated; all rows belong to one weight matrix, so the CTA-pair GEMM is used

@@ -275,6 +275,8 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
 // maxima, watch the arrival words and post each scale on a shared-memory board, where the
 // consumers find it -- one reader per tensor and CTA, because thousands of readers of one
 // address queue up at its L2 slice.
+// For small tensors the grid is cut into `split` sets of CTAs and tensor t goes to set t mod split,
+// so that a CTA's share stays a few chunks long.
 // `pair` holds {amax bits, arrivals} per tensor, zero on entry.  Waits are bounded; a warp that
 // gives up raises a flag that stops the CTA, and NaN is written to the scales not yet posted.
 // ---------------------------------------------------------------------------
@@ -350,7 +352,6 @@ struct RingItems {
     return true;
   }
 };
-
 
 __global__ void __launch_bounds__(kRingThreads, 1)
 fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t tensor_stride, int n_tensors_all,

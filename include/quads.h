@@ -77,6 +77,11 @@ size_t quads_sf_tiled_bytes(int64_t rows, int64_t K);
  *   gs_out out, float[1]: the per-tensor scale that was used (may be NULL)
  *   workspace  >= quads_quantize_workspace_bytes() bytes
  * rows == 0 is allowed (nothing is written except gs_out = 1 when gs_in is NULL).
+ * With gs_in == NULL the kernel is one cooperative launch whose CTAs meet at a
+ * counter once the tensor's amax is complete; that wait is bounded (about two
+ * seconds).  If it ever gives up the call still ends, q and sf are unspecified
+ * and gs_out[0] = NaN says so (pass gs_out to be able to tell); the same holds
+ * for quads_fake_quant_activations.  With gs_in given there is no wait at all.
  * A tensor holds fewer than 2^31 scale blocks (rows * K / 16), else QUADS_ERR_SHAPE;
  * the same limit applies to every tensor of quads_fake_quant_weights.
  */
@@ -207,7 +212,13 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
  * `cuda_stream` and can be captured into a CUDA graph (make one ordinary call
  * first: kernel attributes are set on first use).  Device-side waits are bounded;
  * one that gives up writes QUADS_ERR_TIMEOUT to a status word in the workspace,
- * read with quads_moe_async_status().
+ * read with quads_moe_async_status().  Every call resets that word on its stream
+ * before its first kernel: poll after each call whose status matters.
+ * One side stream per device serves all callers: calls on one device are
+ * serialised on the host by a lock while they enqueue, and a CUDA-graph capture
+ * of a call must not overlap, in time, other MoE calls on the same device (they
+ * would enqueue into the capturing side stream).  The timing and trace aids
+ * below keep process-wide state and are not thread-safe.
  */
 typedef struct {
   int32_t T, H, I, E, topk;
@@ -277,6 +288,21 @@ quads_status quads_moe_last_kernel_ms(float* gemm1_ms /* host */, float* gemm2_m
  */
 quads_status quads_moe_set_stage_trace(int32_t enable);
 int32_t quads_moe_get_stage_trace(const char** names /* host */, float* ms /* host */, int32_t cap);
+
+/*
+ * Test hook (no counterpart in the paper): exercises the give-up path of a
+ * bounded device-side wait without faulting or hanging anything.  It sets the
+ * bound, in SM clock cycles, of the wait in which the CTAs of
+ * quads_quantize_nvfp4 / quads_fake_quant_activations (and of
+ * quads_fake_quant_weights when it takes the same kernel: one tensor, or
+ * tensors above 32 MB) meet at a tensor's arrival counter in global memory, and
+ * a surplus of arrivals to expect that nothing will ever deliver.  With a
+ * surplus > 0 every such wait runs out after `clock_cycles`: the call still
+ * completes, its outputs are unspecified and gs_out = NaN marks them.
+ * clock_cycles <= 0 and extra_arrivals <= 0 restore the defaults (about two
+ * seconds, no surplus).  Process-wide; meant for tests only.
+ */
+void quads_debug_set_quantize_wait(int64_t clock_cycles, int32_t extra_arrivals);
 
 /* Number of kernels the last quads_* call on this host thread enqueued. */
 int32_t quads_last_launch_count(void);

@@ -22,7 +22,9 @@ where marked:
     W X~ = W Q_A(X) - W (M_S (.) Q_A(dX_q)), both terms W4A4 products.
 Pinned: brute-force routing/sort on tiny inputs, float64 triple loop on tiny
 shapes, the exact-integer special case, linearity, E=1/top-1 reducing to the
-dense projection.
+dense projection; the `h_override` and forced-selection branches (used by the
+staged comparison of an implementation) against explicit loops and a
+brute-force re-mask.
 """
 import numpy as np
 

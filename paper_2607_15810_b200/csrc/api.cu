@@ -202,6 +202,7 @@ struct SideStream {
   bool ok = false;
 };
 std::mutex g_side_mu;
+// Call with g_side_mu held (the per-device objects are created on first use).
 SideStream* side_stream() {
   static SideStream per_device[64];
   static const bool disabled = [] { const char* e = getenv("QUADS_NO_OVERLAP"); return e && e[0] == '1'; }();
@@ -218,6 +219,22 @@ SideStream* side_stream() {
   }
   return &s;
 }
+
+// Joins the side stream back into the caller's stream when the scope is left before the regular
+// join (an error return between fork and join): without it the side stream would stay forked
+// and, under stream capture, the captured graph would be left with an unjoined branch.
+struct SideJoinGuard {
+  SideStream* side = nullptr;
+  cudaStream_t main = nullptr;
+  bool joined = true;
+  void arm(SideStream* s, cudaStream_t st) { side = s; main = st; joined = false; }
+  void join() {
+    if (joined || !side) return;
+    joined = true;
+    if (cudaEventRecord(side->join, side->stream) == cudaSuccess) cudaStreamWaitEvent(main, side->join, 0);
+  }
+  ~SideJoinGuard() { join(); }
+};
 
 // GEMM variant of a call.  1: single-CTA tiles of 128 x 256; 2: CTA pairs computing 256 x 256
 // tiles with cta_group::2 MMAs: about 7 % (first projection) / 5 % (second) faster per tile, but
@@ -279,6 +296,16 @@ size_t quads_fake_quant_workspace_bytes(int64_t n_tensors) {
   return align_up((size_t)(n_tensors > 0 ? n_tensors : 1) * 8, 256);
 }
 int32_t quads_last_launch_count(void) { return g_launch_count; }
+
+// Bound of the per-tensor arrival wait of fused_quantize_kernel in SM clock cycles (about two
+// seconds), and a test-only surplus of expected arrivals (see quads_debug_set_quantize_wait).
+static std::atomic<long long> g_quant_wait_cycles{4000000000ll};
+static std::atomic<int> g_quant_extra_arrivals{0};
+
+void quads_debug_set_quantize_wait(int64_t clock_cycles, int32_t extra_arrivals) {
+  g_quant_wait_cycles.store(clock_cycles > 0 ? (long long)clock_cycles : 4000000000ll);
+  g_quant_extra_arrivals.store(extra_arrivals > 0 ? (int)extra_arrivals : 0);
+}
 
 static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t rows, int64_t K, int64_t ld,
                                     int64_t tensor_stride, const float* gs_in, void* fq, uint8_t* q, uint8_t* sf,
@@ -358,8 +385,10 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   int grid = di.sm_count * blocks_per_sm;
   if (want < grid) grid = (int)want;
   if (grid < n_groups) grid = n_groups;
+  long long wait_cycles = g_quant_wait_cycles.load();
+  int extra_arrivals = g_quant_extra_arrivals.load();
   void* args[] = {&xp, &rows, &K, &ld, &tensor_stride, &nt, &gs_in, &amax_bits, &counters, &q, &sf, &fqp,
-                  &gs_out, &tiled, &sf_stride, &n_groups};
+                  &gs_out, &tiled, &sf_stride, &n_groups, &wait_cycles, &extra_arrivals};
   QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fused_quantize_kernel), dim3(grid), dim3(256),
                                             args, 0, st));
   note_launch();
@@ -563,13 +592,20 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   trace_mark("memset", st);
 
   // ---- routing and dispatch order: on a side stream, next to the activation chain below
+  // (declared in this order: on an early return the guard joins first, then the lock is released)
   std::unique_lock<std::mutex> side_lock(g_side_mu, std::defer_lock);
-  SideStream* side = (dense || g_trace.enabled) ? nullptr : side_stream();
+  SideJoinGuard side_guard;
+  SideStream* side = nullptr;
+  if (!dense && !g_trace.enabled) {
+    side_lock.lock();                       // event record / wait pairs of two host threads must not interleave
+    side = side_stream();
+    if (!side) side_lock.unlock();
+  }
   cudaStream_t rs = st;
   if (side) {
-    side_lock.lock();                       // event record / wait pairs of two host threads must not interleave
     QUADS_CUDA_OK(cudaEventRecord(side->fork, st));
     QUADS_CUDA_OK(cudaStreamWaitEvent(side->stream, side->fork, 0));
+    side_guard.arm(side, st);
     rs = side->stream;
   }
   if (dense) {
@@ -652,7 +688,6 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
       QUADS_CUDA_OK(cudaStreamWaitEvent(side->stream, side->mid, 0));
       QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3(scatter_grid), dim3(256), (size_t)(0), side->stream, T, H, 1, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
     }
-    QUADS_CUDA_OK(cudaEventRecord(side->join, side->stream));
   }
   if (nsel13 > 0) {
     s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
@@ -662,7 +697,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   trace_mark("select13", st);
   if (side) {
-    QUADS_CUDA_OK(cudaStreamWaitEvent(st, side->join, 0));
+    side_guard.join();
     side_lock.unlock();
   }
   {

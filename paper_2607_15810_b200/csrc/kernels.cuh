@@ -19,7 +19,8 @@ __global__ void amax_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t 
 __global__ void fused_quantize_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
                                       int n_tensors, const float* gs_in, uint32_t* amax_bits, uint32_t* counters,
                                       uint8_t* q, uint8_t* sf, uint16_t* fq, float* gs_out, int sf_tiled,
-                                      int64_t sf_tensor_stride, int n_groups);
+                                      int64_t sf_tensor_stride, int n_groups, long long wait_cycles,
+                                      int extra_arrivals);
 // Fake-quant of a batch of tensors through shared-memory rings of bulk copies (one CTA per SM,
 // four groups of 7 consumer warps + 1 producer warp, one ring of 14 KB stages per group).
 constexpr int kRingThreads = 1024;

@@ -144,7 +144,7 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
                       int n_tensors, const float* __restrict__ gs_in, uint32_t* __restrict__ amax_bits,
                       uint32_t* __restrict__ counters, uint8_t* __restrict__ q, uint8_t* __restrict__ sf,
                       uint16_t* __restrict__ fq, float* __restrict__ gs_out, int sf_tiled, int64_t sf_tensor_stride,
-                      int n_groups) {
+                      int n_groups, long long wait_cycles, int extra_arrivals) {
   const int group = blockIdx.x % n_groups;
   const int rank = blockIdx.x / n_groups;
   const int gsize = ((int)gridDim.x - group + n_groups - 1) / n_groups;
@@ -201,9 +201,10 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
         // bounded wait for the rest of the group (cooperative launch: all CTAs are resident)
         const long long t0 = clock64();
         bool gave_up = false;
-        while (atomicAdd(counters + t, 0u) < (uint32_t)gsize) {
+        // (extra_arrivals is zero except under the test hook that makes this wait run out)
+        while (atomicAdd(counters + t, 0u) < (uint32_t)(gsize + extra_arrivals)) {
           __nanosleep(64);
-          if (clock64() - t0 > 4000000000ll) { gave_up = true; break; }
+          if (clock64() - t0 > wait_cycles) { gave_up = true; break; }
         }
         __threadfence();
         // (the count only grows, so if one CTA of the group gives up on it, all do: NaN marks the tensor)
@@ -307,12 +308,17 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// One aligned 8-byte load of a tensor's {amax bits, arrivals} pair.  A CTA publishes its maximum,
-// fences, then counts itself in, and the load is a single access to one L2 sector, so a pair that
-// shows all arrivals also shows the final maximum.
-__device__ __forceinline__ uint64_t ld_relaxed_u64(const void* p) {
-  uint64_t v;
-  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+// Acquire load of a tensor's arrival word.  A CTA publishes its maximum (atomicMax), fences, then
+// counts itself in: once this load shows every arrival, a later load of the amax word returns the
+// final maximum.
+__device__ __forceinline__ uint32_t ld_acquire_u32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
@@ -420,9 +426,8 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
     uint64_t keep, stream;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(keep));
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(stream));
-    const uint64_t* words = reinterpret_cast<const uint64_t*>(pair);
     int watch = group;                                           // the tensor whose arrival word this producer reads next
-    uint64_t seen = 0;
+    uint32_t seen = 0;
     bool asked = false;
     long long asked_at = 0;
     // One look at the arrival word of tensor `watch`; posts the scale once every CTA has arrived.
@@ -443,14 +448,15 @@ fake_quant_ring_kernel(const uint16_t* __restrict__ x, int64_t nblk, int64_t ten
       }
       if (watch >= n_tensors) return;
       if (asked && clock64() - asked_at < 2000) return;
-      if (asked && (uint32_t)(seen >> 32) == (uint32_t)ctas_per_tensor) {
-        if (gs_out && cta_in_set == 0) gs_out[glob(watch)] = gs_from_amax_bits((uint32_t)seen);
-        sh->board[watch & (kRingBoard - 1)] = ((unsigned long long)((uint32_t)watch + 1u) << 32) | (uint32_t)seen;
+      if (asked && seen == (uint32_t)ctas_per_tensor) {
+        const uint32_t amax_b = ld_relaxed_u32(pair + 2 * glob(watch));   // ordered after the acquire load above
+        if (gs_out && cta_in_set == 0) gs_out[glob(watch)] = gs_from_amax_bits(amax_b);
+        sh->board[watch & (kRingBoard - 1)] = ((unsigned long long)((uint32_t)watch + 1u) << 32) | amax_b;
         watch += kRingGroups;
         asked = false;
         if (watch >= n_tensors) return;
       }
-      seen = ld_relaxed_u64(words + glob(watch));
+      seen = ld_acquire_u32(pair + 2 * glob(watch) + 1);
       asked = true;
       asked_at = clock64();
     };

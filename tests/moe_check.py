@@ -129,13 +129,59 @@ def check_moe(res, x, logits, w13o, w2o, topk, nsel13, nsel2, a2_gs, renormalize
     return report
 
 
+def sample_plan(ids, offsets, topk, hot_experts, n_tokens, tail_experts, seed):
+    """Which outputs of a full-size layer the oracle recomputes one by one.
+    Tokens: a seeded random order, taken greedily until every expert that has
+    rows is hit by a sampled token, then topped up to n_tokens; all rows of a
+    sampled token are checked (h) and so is its row of `out`.  Extra dispatched
+    rows (h only): the first and the last row of every expert, three rows of
+    the first tile and the first / last row of the last tile of every hot
+    expert, and one row in every 128-row tile of the last `tail_experts`
+    experts (the tiles the persistent kernels take in their last wave)."""
+    T = ids.shape[0]
+    E = offsets.size - 1
+    rng = np.random.default_rng(seed)
+    order = rng.permutation(T)
+    need = {e for e in range(E) if offsets[e + 1] > offsets[e]}
+    tokens = []
+    for t in order:
+        hit = need & {int(e) for e in ids[t]}
+        if hit:
+            tokens.append(int(t))
+            need -= hit
+        if not need:
+            break
+    for t in order:
+        if len(tokens) >= n_tokens:
+            break
+        if int(t) not in tokens:
+            tokens.append(int(t))
+    rows = set()
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi == lo:
+            continue
+        rows.update((lo, hi - 1))
+        if e < hot_experts:
+            rows.update(r for r in (lo + 64, lo + 127) if r < hi)
+            rows.add(lo + ((hi - lo - 1) // 128) * 128)
+        if e >= E - tail_experts:
+            rows.update(range(lo + int(rng.integers(0, 128)) % max(1, min(128, hi - lo)), hi, 128))
+    return sorted(tokens), sorted(rows)
+
+
 def check_moe_sampled(res, x, logits, shape, w13_bf16_of, w2_bf16_of, nsel13, nsel2, a2_gs,
-                      sample_tokens, renormalize=True):
+                      n_tokens=64, n_features=96, n_columns=128, tail_experts=8, renormalize=True, seed=99):
     """Full-size variant: everything that is cheap on the CPU is compared in
     full and bit-exactly (routing, dispatch, Q_A(x), selection, residual, and the
     requantization of the implementation's own h); the two GEMMs are compared on
-    sampled outputs the oracle computes one by one: every dispatched row of the
-    sampled tokens for h, and the sampled tokens' rows of `out`.
+    sampled outputs the oracle computes one by one (see sample_plan): for every
+    sampled dispatched row, `n_features` features of h (every 128-feature tile
+    of the first projection is hit) against the float64 contraction; for every
+    sampled token, `n_columns` columns of `out` (every 256-column tile hit)
+    against the float64 contraction of the implementation's own quantized h.
+    Each expert's weights are quantized by the oracle once: the per-tensor scale
+    from the whole tensor, codes and block scales for the sampled rows only.
     w13_bf16_of / w2_bf16_of: callables expert -> bf16 torch weight [N, K]."""
     report = {}
     xf = f32(x)
@@ -165,50 +211,86 @@ def check_moe_sampled(res, x, logits, shape, w13_bf16_of, w2_bf16_of, nsel13, ns
         assert np.array_equal(res["r2sf"].cpu().numpy(), site2["r_sf"]), "residual-of-h scales differ"
     report["site2_bit_exact"] = True
     # ---- sampled GEMM outputs
+    tokens, extra_rows = sample_plan(ids, offsets, topk, shape.hot_experts, n_tokens, tail_experts, seed)
     inv = np.empty(T * topk, dtype=np.int64)
     inv[perm] = np.arange(T * topk)
-    xt = R.reconstruct_real(site13)
-    xa = (np.abs(Q.dequantize_real(site13["codes"], site13["sf"], site13["gs"]))
-          + np.abs(Q.dequantize_real(site13["r_codes"], site13["r_sf"], site13["r_gs"])))
+    tok_rows = {int(inv[t * topk + s]): (t, s) for t in tokens for s in range(topk)}
+    rows = sorted(set(extra_rows) | set(tok_rows))
+    row_expert = np.searchsorted(offsets, np.asarray(rows), side="right") - 1
+    tok_of = perm // topk
+    rng = np.random.default_rng(seed + 1)
+
+    def spread(n_total, tile, n_pick):
+        """n_pick indices of range(n_total): the first, the last, and a seeded
+        choice with every `tile`-sized tile represented."""
+        per = max(1, n_pick // max(1, n_total // tile))
+        pick = {0, n_total - 1}
+        for t0 in range(0, n_total, tile):
+            pick.update(int(v) for v in t0 + rng.choice(min(tile, n_total - t0), size=min(per, n_total - t0), replace=False))
+        return np.array(sorted(pick), dtype=np.int64)
+
+    cols = spread(H, 256, n_columns)
+    xt_all = R.reconstruct_real(site13)
+    xa_all = (np.abs(Q.dequantize_real(site13["codes"], site13["sf"], site13["gs"]))
+              + np.abs(Q.dequantize_real(site13["r_codes"], site13["r_sf"], site13["r_gs"])))
     out_gpu = f32(res["out"]).astype(np.float64)
-    worst_h, worst_o = 0.0, 0.0
-    experts = sorted({int(e) for t in sample_tokens for e in ids[t]})
-    wcache = {}
-    for e in experts:
-        wcache[e] = (oracle_weights(w13_bf16_of(e)[None]), oracle_weights(w2_bf16_of(e)[None]))
-    for t in sample_tokens:
-        o64 = np.zeros(H)
-        oad = np.zeros(H)
-        for s in range(topk):
-            e = int(ids[t, s])
-            row = inv[t * topk + s]
-            w13o, w2o = wcache[e]
-            w = Q.dequantize_real(w13o["codes"][0], w13o["sf"][0], w13o["gs"][0])
-            g = w @ xt[t]
-            gad = np.abs(w) @ xa[t]
-            gate, up = g[:I], g[I:]
-            sig = 1.0 / (1.0 + np.exp(-gate))
-            h64 = gate * sig * up
-            dsilu = sig * (1.0 + gate * (1.0 - sig))
-            dg, du = GEMM_RTOL * gad[:I], GEMM_RTOL * gad[I:]
-            tol_h = (np.abs(dsilu * up) * dg + np.abs(gate * sig) * du + dg * du * 2
-                     + (BF16_ULP + 1e-5) * np.abs(h64) + 1e-30)
-            worst_h = max(worst_h, float((np.abs(h_gpu[row] - h64) / tol_h).max()))
-            # second projection on the implementation's own quantized h
-            one = {k: (v[row:row + 1] if isinstance(v, np.ndarray) and v.ndim == 2 and v.shape[0] == h_gpu.shape[0] else v)
+    o64 = {t: np.zeros(cols.size) for t in tokens}
+    oad = {t: np.zeros(cols.size) for t in tokens}
+    worst_h, n_h, experts_hit, tiles_hit = 0.0, 0, set(), set()
+    for e in sorted(set(int(v) for v in row_expert)):
+        mine = [r for r, re_ in zip(rows, row_expert) if re_ == e]
+        experts_hit.add(e)
+        w13 = f32(w13_bf16_of(e))                               # [2I, H] bf16 values
+        feats = spread(I, 128, n_features)
+        gs13 = Q.tensor_global_scale(w13)                      # per-tensor scale: from the WHOLE tensor
+        sub = np.concatenate([w13[feats], w13[I + feats]])     # gate rows, then up rows of the sampled features
+        c13, s13, _ = Q.quantize(sub, gs13)
+        wd = Q.dequantize_real(c13, s13, gs13)
+        toks = tok_of[np.asarray(mine)]
+        g = xt_all[toks] @ wd.T
+        gad = xa_all[toks] @ np.abs(wd).T
+        nf = feats.size
+        gate, up = g[:, :nf], g[:, nf:]
+        sig = 1.0 / (1.0 + np.exp(-gate))
+        h64 = gate * sig * up
+        dsilu = sig * (1.0 + gate * (1.0 - sig))
+        dg, du = GEMM_RTOL * gad[:, :nf], GEMM_RTOL * gad[:, nf:]
+        tol_h = (np.abs(dsilu * up) * dg + np.abs(gate * sig) * du + dg * du * 2
+                 + (BF16_ULP + 1e-5) * np.abs(h64) + 1e-30)
+        got = h_gpu[np.asarray(mine)][:, feats]
+        worst_h = max(worst_h, float((np.abs(got - h64) / tol_h).max()))
+        n_h += got.size
+        tiles_hit.update((e, (r - int(offsets[e])) // 128) for r in mine)
+        # second projection on the implementation's own quantized h, for the rows of sampled tokens
+        mine_tok = [r for r in mine if r in tok_rows]
+        if mine_tok:
+            w2 = f32(w2_bf16_of(e))                             # [H, I]
+            gs2 = Q.tensor_global_scale(w2)
+            c2, s2, _ = Q.quantize(w2[cols], gs2)
+            w2d = Q.dequantize_real(c2, s2, gs2)
+            idx = np.asarray(mine_tok)
+            one = {k: (v[idx] if isinstance(v, np.ndarray) and v.ndim == 2 and v.shape[0] == h_gpu.shape[0] else v)
                    for k, v in site2.items()}
-            ht = R.reconstruct_real(one)[0]
+            ht = R.reconstruct_real(one)
             ha = (np.abs(Q.dequantize_real(one["codes"], one["sf"], one["gs"]))
-                  + np.abs(Q.dequantize_real(one["r_codes"], one["r_sf"], one["r_gs"])))[0]
-            w2 = Q.dequantize_real(w2o["codes"][0], w2o["sf"][0], w2o["gs"][0])
-            o64 += float(wts[t, s]) * (w2 @ ht)
-            oad += float(wts[t, s]) * (np.abs(w2) @ ha)
-        tol_o = gemm_tol(oad, o64) + 4e-5 * oad
-        worst_o = max(worst_o, float((np.abs(out_gpu[t] - o64) / tol_o).max()))
+                  + np.abs(Q.dequantize_real(one["r_codes"], one["r_sf"], one["r_gs"])))
+            y, ya = ht @ w2d.T, ha @ np.abs(w2d).T
+            for k, r in enumerate(mine_tok):
+                t, s_ = tok_rows[r]
+                o64[t] += float(wts[t, s_]) * y[k]
+                oad[t] += float(wts[t, s_]) * ya[k]
+    worst_o = 0.0
+    for t in tokens:
+        tol_o = gemm_tol(oad[t], o64[t]) + 4e-5 * oad[t]
+        worst_o = max(worst_o, float((np.abs(out_gpu[t][cols] - o64[t]) / tol_o).max()))
     report["h_max_err_over_tol"] = worst_h
     report["out_max_err_over_tol"] = worst_o
-    report["sampled_tokens"] = len(sample_tokens)
-    report["sampled_experts"] = len(experts)
+    report["sampled_tokens"] = len(tokens)
+    report["sampled_rows"] = len(rows)
+    report["sampled_experts"] = len(experts_hit)
+    report["sampled_row_tiles"] = len(tiles_hit)
+    report["h_values_checked"] = n_h
+    report["out_values_checked"] = len(tokens) * int(cols.size)
     assert worst_h <= 1.0, "h outside tolerance: %g" % worst_h
     assert worst_o <= 1.0, "out outside tolerance: %g" % worst_o
     return report

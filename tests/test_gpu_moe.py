@@ -76,6 +76,68 @@ def test_dense_exact_integer_case(B):
     assert np.array_equal(got, MC.f32(torch.from_numpy(want).to(torch.bfloat16)).astype(np.float64))
 
 
+def test_dense_at_the_size_where_cta_pairs_are_chosen(B):
+    """From 1024 rows per weight matrix the call takes the CTA-pair kernel (256 x 256 tiles,
+    cta_group::2) on its own; compared element by element with the oracle, ragged last pair."""
+    x, w = synth.dense_inputs(seed=9, T=2300, K=1024, N=640)
+    ratio = _dense_case(B, x, w, 512)
+    print("cta-pair dense 2300x1024x640: worst err / tol = %.3f" % ratio)
+
+
+def _sweep_operands():
+    """Operands in which every finite non-negative E4M3 scale code and every E2M1 nibble occurs on
+    both sides of the tensor-core product, laid out so that a single wrong decode shows: weight row
+    n is non-zero in block n only, hence out[t, n] is the 16-term product of activation block
+    (t, n) and weight block n, all terms of one sign.  Values are exactly representable (<= 6
+    significant bits), so the quantizers reproduce the chosen codes."""
+    mags = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float64)
+    sf = F.E4M3_MAGNITUDES[:127].astype(np.float64)             # codes 0x00 .. 0x7E
+    T, NB = 128, 128
+    K = NB * 16
+    a_gs, w_gs = 2.0 ** -6, 2.0 ** -10
+    i = np.arange(16)
+    sgn = np.where(i < 8, 1.0, -1.0)
+    x = np.zeros((T, K))
+    w = np.zeros((NB, K))
+    for n in range(NB):
+        w[n, 16 * n:16 * n + 16] = sgn * mags[(i + n) % 8] * sf[n % 127] * w_gs
+        for t in range(T):
+            x[t, 16 * n:16 * n + 16] = sgn * mags[(i + t) % 8] * sf[(t + n) % 127] * a_gs
+    xb, wb = torch.from_numpy(x).to(torch.bfloat16), torch.from_numpy(w).to(torch.bfloat16)
+    assert np.array_equal(xb.to(torch.float64).numpy(), x) and np.array_equal(wb.to(torch.float64).numpy(), w)
+    return xb, wb, np.float32(a_gs), np.float32(w_gs)
+
+
+def test_tensor_cores_decode_every_scale_code_and_every_nibble(B):
+    xb, wb, a_gs, w_gs = _sweep_operands()
+    wo = MC.oracle_weights(wb[None])
+    assert wo["gs"][0] == w_gs                                  # amax = 6 * 448 * w_gs
+    o = M.dense_w4a4_rac(MC.f32(xb), wo["codes"][0], wo["sf"][0], wo["gs"][0], 0, a_gs=a_gs)
+    # the sweep really covers the code space on both sides
+    assert set(o["site"]["sf"].reshape(-1).tolist()) == set(range(127))
+    assert set(np.diag(wo["sf"][0][:, :128]).tolist()) == set(range(127))
+    w_blocks = np.stack([wo["codes"][0][n, 16 * n:16 * n + 16] for n in range(128)])
+    for side in (o["site"]["codes"], w_blocks):
+        assert set(side.reshape(-1).tolist()) >= set(range(1, 8)) | set(range(9, 16))
+    wq = B.fake_quant_weights(wb.unsqueeze(0).cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    assert np.array_equal(wq["q"].cpu().numpy(), wo["q"])
+    res = B.dense_w4a4_rac(xb.cuda(), wq, 0, a_gs=torch.tensor([float(a_gs)]).cuda(), export=True)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    MC.check_site1(res, dict(site13=o["site"]), 0, {})
+    got = MC.f32(res["out"]).astype(np.float64)
+    # all products of an output have one sign: sum|a b| = |y|, so the bound is 2e-3 |y| + one bf16 ulp,
+    # while a mis-decoded scale byte or nibble changes y by at least 1/16 of itself
+    assert np.allclose(o["absdot"], np.abs(o["y64"]), rtol=1e-12)
+    ratio = float((np.abs(got - o["y64"]) / MC.gemm_tol(o["absdot"], o["y64"])).max())
+    assert ratio <= 1.0, ratio
+    exact = float((got == MC.f32(torch.from_numpy(o["y64"]).to(torch.bfloat16))).mean())
+    print("scale/nibble sweep: worst err / tol = %.3f, outputs equal to the rounded exact value: %.4f" % (ratio, exact))
+    # with every channel compensated nothing changes: the residual of exactly representable values is zero
+    res_k = B.dense_w4a4_rac(xb.cuda(), wq, xb.shape[1], a_gs=torch.tensor([float(a_gs)]).cuda())
+    assert torch.equal(res_k["out"], res["out"])
+
+
 def _moe_small(B, name, f13, f2, renorm, shape=None):
     sh = shape if shape is not None else synth.MOE_SHAPES[name]
     x, _ = synth.activations(sh)
@@ -93,11 +155,10 @@ def _moe_small(B, name, f13, f2, renorm, shape=None):
     torch.cuda.synchronize()
     assert B.moe_async_status(res["workspace"]) == 0
     rep = MC.check_moe(res, x, lg, w13o, w2o, sh.topk, nsel13, nsel2, a2, renormalize=renorm)
-    # the export-free call gives the same output bits for everything but the atomics' order
+    # the export-free call gives the same output bits (every reduction runs in a fixed order)
     res2 = B.moe_w4a4_rac(x.cuda(), lg.cuda(), gw13, gw2, sh.topk, nsel13, nsel2, torch.tensor([a2]).cuda(),
                           renormalize=renorm)
-    d = (MC.f32(res2["out"]) - MC.f32(res["out"]))
-    assert np.abs(d).max() <= 2.0 ** -6 * np.abs(MC.f32(res["out"])).max()
+    assert torch.equal(res2["out"], res["out"])
     return rep
 
 
@@ -199,14 +260,19 @@ def test_moe_full_size_sampled(B, name, variant):
         ids = res["ids"].cpu().numpy()
         share = float((ids < sh.hot_experts).mean())
         assert abs(share - sh.hot_share) <= 0.005
-    n_tok = 2 if name == "large" else 3
-    rng = np.random.default_rng(99)
-    tokens = sorted(int(t) for t in rng.choice(sh.T, n_tok, replace=False))
+    # >= 512 dispatched rows over every expert, the first and last tile of every hot expert and the last
+    # wave of tiles; the variants other than the benchmarked one take a lighter plan (they share the kernels)
+    heavy = variant == "both"
     rep = MC.check_moe_sampled(res, x, lg, sh,
                                lambda e: synth.expert_weights(sh, "w13", [e])[0],
                                lambda e: synth.expert_weights(sh, "w2", [e])[0],
-                               nsel13, nsel2, a2, tokens)
+                               nsel13, nsel2, a2, n_tokens=64 if heavy else 16, n_features=96 if heavy else 48,
+                               n_columns=128 if heavy else 64, tail_experts=8 if heavy else 2)
     assert rep["h_max_err_over_tol"] <= 1 and rep["out_max_err_over_tol"] <= 1
+    assert rep["sampled_experts"] == sh.E
+    if heavy:
+        assert rep["sampled_rows"] >= 512 and rep["sampled_tokens"] >= 64
+    print(name, variant, rep)
     for k in ("xq", "rq", "h", "hq", "r2q"):
         res.pop(k)
 

@@ -208,3 +208,64 @@ def test_dequantize_gives_the_trainers_fake_quant_bit_for_bit(B, n, N, K):
     for i in range(n):
         dec = Q.dequantize_bf16(F.unpack_nibbles(lin["q"][i].cpu().numpy()), lin["sf"][i].cpu().numpy(), lin["gs"][i].item())
         assert np.array_equal(F.bf16_bits(dec), F.bf16_bits(_f32(d_lin[i])))
+
+
+@pytest.mark.parametrize("N,K", [(3072, 4096), (4096, 1536)])
+def test_aqat_layer_batch_at_full_size_against_the_oracle_on_sampled_tensors(B, N, K):
+    """The fake-quant + weight-sync workload in the launch configuration the benchmark times: 128
+    expert tensors of one shape in one call (one cooperative launch of the ring kernel).  The batch
+    is drawn on the device (seeded); the first, the last and three tensors in between are copied
+    back and compared bit for bit with the oracle; trainer == rollout is checked on every tensor."""
+    n = 128
+    g = torch.Generator(device="cuda").manual_seed(4 * 1000003 + N)
+    w = torch.empty(n, N, K, dtype=torch.bfloat16, device="cuda")
+    for e0 in range(0, n, 16):
+        w[e0:e0 + 16] = (torch.randn(16, N, K, device="cuda", generator=g) * 0.015).to(torch.bfloat16)
+    r = B.fake_quant_weights(w)
+    torch.cuda.synchronize()
+    assert B.last_launch_count() == 1
+    assert torch.isfinite(r["gs"]).all()
+    # Eq. weight-qdq-align on all 128 tensors: decoding the packed bytes gives the trainer's bf16 bits
+    dec = B.dequantize_nvfp4(r["q"], r["sf"], r["gs"], N, K)
+    assert torch.equal(dec.view(torch.int16), r["w_fq"].view(torch.int16))
+    del dec
+    for i in (0, 41, 77, 126, 127):
+        wf_o, q_o, sf_o, gs_o = Q.fake_quant_weights(_f32(w[i:i + 1]))
+        assert np.array_equal(r["gs"][i:i + 1].cpu().numpy(), gs_o), i
+        assert np.array_equal(r["q"][i].cpu().numpy(), q_o[0]), i
+        assert np.array_equal(r["sf"][i].cpu().numpy(), sf_o[0]), i
+        assert np.array_equal(F.bf16_bits(_f32(r["w_fq"][i])), F.bf16_bits(wf_o[0])), i
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_harmless(B):
+    """Failure detection without a fault: the test hook makes the arrival wait of the quantize kernel
+    expect one arrival more than there are CTAs and shortens its bound to about a millisecond.  The
+    call must still end, mark its scale as NaN, and leave the library usable: the next ordinary call
+    is bit-exact against the oracle."""
+    x = _bf16((1, 16), 31, 2.0).cuda()
+    lib = B.lib
+    lib.quads_debug_set_quantize_wait.restype = None
+    lib.quads_debug_set_quantize_wait.argtypes = [B.C.c_int64, B.C.c_int32]
+    lib.quads_debug_set_quantize_wait(2_000_000, 1)
+    try:
+        q, sf, gs = B.quantize_nvfp4(x)
+        torch.cuda.synchronize()
+        assert torch.isnan(gs).all()
+        xf, g2 = B.fake_quant_activations(x)
+        torch.cuda.synchronize()
+        assert torch.isnan(g2).all()
+    finally:
+        lib.quads_debug_set_quantize_wait(0, 0)
+    big = _bf16((333, 2048), 3, 3.0)
+    q, sf, gs = B.quantize_nvfp4(big.cuda())
+    c_o, s_o, g_o = Q.quantize(_f32(big))
+    assert np.float32(gs.item()) == g_o and np.array_equal(sf.cpu().numpy(), s_o)
+    assert np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o))
+    # with a supplied scale there is no wait at all, hook or not
+    lib.quads_debug_set_quantize_wait(2_000_000, 1)
+    try:
+        q2, sf2, g3 = B.quantize_nvfp4(big.cuda(), gs=gs)
+        torch.cuda.synchronize()
+    finally:
+        lib.quads_debug_set_quantize_wait(0, 0)
+    assert torch.equal(q2, q) and torch.equal(sf2, sf) and g3.item() == gs.item()

@@ -240,3 +240,164 @@ def test_moe_two_experts_against_explicit_loops():
     assert np.array_equal(out["out"], F.bf16_round(out["out64"]))
     # site-2 statistics run over all dispatched rows at once
     assert out["site2"]["codes"].shape == (18, 16) and out["site2"]["sel"].size == 8
+
+
+def _two_expert_case():
+    shape = synth.MoEShape("t", 23, 9, 32, 3, 2, 16, 0.05, 1, 3.0, 10.0)
+    x, _ = synth.activations(shape)
+    x = x.to(torch.float32).numpy()
+    logits = synth.router_logits(shape).numpy()
+    return x, logits, _tiny_weights(3, 32, 32, 51), _tiny_weights(3, 32, 16, 52), np.float32(0.003)
+
+
+def _second_half_by_loops(out, ht, w2):
+    """out[t] = sum over the token's slots of weight * W2_e h~[row], explicit loops."""
+    T, topk = out["ids"].shape
+    inv = np.empty(T * topk, int)
+    inv[out["perm"]] = np.arange(T * topk)
+    want = np.zeros((T, w2["codes"].shape[1]))
+    for t in range(T):
+        for s in range(topk):
+            e = int(out["ids"][t, s])
+            w2e = _scalar_dequant(w2["codes"][e], w2["sf"][e], w2["gs"][e])
+            want[t] += float(out["weights"][t, s]) * _triple_loop([ht[inv[t * topk + s]].tolist()], w2e.tolist())[0]
+    return want
+
+
+def test_h_override_replays_and_replaces_the_second_half():
+    """The staged comparison of an implementation runs the layer's second half
+    on that implementation's own h.  Feeding the oracle its own h must change
+    nothing; feeding it a perturbed h must give exactly what site-2 RAC and
+    the down projection give for that h."""
+    x, logits, w13, w2, a2 = _two_expert_case()
+    base = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2)
+    same = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, h_override=base["h"])
+    for k in ("codes", "sf", "r_codes", "r_sf", "sel", "scores", "residual"):
+        assert np.array_equal(same["site2"][k], base["site2"][k]), k
+    assert same["site2"]["gs"] == base["site2"]["gs"] and same["site2"]["r_gs"] == base["site2"]["r_gs"]
+    assert np.array_equal(same["out64"], base["out64"]) and np.array_equal(same["out_absdot"], base["out_absdot"])
+    assert np.array_equal(same["out"], base["out"])
+    # one bf16 ulp up on a few elements (and one sign flip): a different, equally valid h
+    hp = base["h"].copy()
+    bits = F.bf16_bits(hp).astype(np.uint32)
+    for (i, j) in ((0, 0), (3, 7), (11, 15), (17, 2)):
+        bits[i, j] += 1
+    bits[5, 5] ^= 0x8000
+    hp = (bits << 16).view(np.float32).reshape(hp.shape)
+    assert np.all(F.bf16_round(hp) == hp) and (hp != base["h"]).sum() >= 4
+    pert = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, h_override=hp)
+    assert np.array_equal(pert["h"], base["h"])               # the oracle's own h is still reported
+    want_site = R.rac(hp, 8, a2)
+    for k in ("codes", "sf", "r_codes", "r_sf", "sel"):
+        assert np.array_equal(pert["site2"][k], want_site[k]), k
+    assert pert["site2"]["gs"] == a2 and pert["site2"]["r_gs"] == a2
+    assert not np.array_equal(pert["site2"]["codes"], base["site2"]["codes"])   # the override is not ignored
+    want = _second_half_by_loops(pert, R.reconstruct_real(want_site), w2)
+    assert np.allclose(pert["out64"], want, rtol=1e-11, atol=1e-14)
+    assert not np.allclose(pert["out64"], base["out64"], rtol=1e-6, atol=0)
+    # the tolerance denominator follows the overriding operands too
+    ha = (np.abs(_scalar_dequant(want_site["codes"], want_site["sf"], a2))
+          + np.abs(_scalar_dequant(want_site["r_codes"], want_site["r_sf"], a2)))
+    absd = np.zeros_like(want)
+    inv = np.empty(18, int)
+    inv[pert["perm"]] = np.arange(18)
+    for t in range(9):
+        for s in range(2):
+            e = int(pert["ids"][t, s])
+            w2e = np.abs(_scalar_dequant(w2["codes"][e], w2["sf"][e], w2["gs"][e]))
+            absd[t] += float(pert["weights"][t, s]) * _triple_loop([ha[inv[t * 2 + s]].tolist()], w2e.tolist())[0]
+    assert np.allclose(pert["out_absdot"], absd, rtol=1e-11)
+
+
+def test_forced_selection_is_a_brute_force_remask():
+    """_force_selection with the site's own set is the identity; with another
+    set it equals clearing, by hand, the unselected channels of the quantized
+    full residual (block scales untouched, everything else unchanged)."""
+    x, _ = _dense()
+    x = x[:24, :64]
+    site = R.rac(x, 16)
+    ident = M._force_selection(x, site, site["sel"])
+    assert set(ident) == set(site)
+    for k, v in site.items():
+        assert np.array_equal(ident[k], v), k
+    other = np.array([63, 0, 17, 5, 40], dtype=np.int32)        # unsorted on purpose
+    forced = M._force_selection(x, site, other)
+    full_c, full_s, full_g = Q.quantize(site["residual"], site["r_gs"])
+    assert full_g == site["r_gs"] == site["gs"]                 # the residual shares its activation's scale
+    want = np.zeros_like(full_c)
+    for j in other:
+        want[:, j] = full_c[:, j]
+    assert np.array_equal(forced["r_codes"], want)
+    assert np.array_equal(forced["sel"], np.sort(other))
+    assert np.array_equal(forced["r_sf"], full_s) and np.array_equal(forced["r_sf"], site["r_sf"])
+    for k in ("codes", "sf", "gs", "residual", "scores", "r_gs"):
+        assert np.array_equal(forced[k], site[k]), k
+    # a forced set that differs from the top-16 changes the reconstruction
+    assert not np.array_equal(R.reconstruct_real(forced), R.reconstruct_real(site))
+
+
+def test_forced_selections_flow_through_the_layer():
+    """moe_forward(forced_sel13 / forced_sel2): with the sets the oracle picks
+    itself nothing changes; with other sets the layer equals the explicit
+    loops run on the re-masked operands."""
+    x, logits, w13, w2, a2 = _two_expert_case()
+    base = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2)
+    same = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, forced_sel13=base["site13"]["sel"],
+                         forced_sel2=base["site2"]["sel"])
+    assert np.array_equal(same["g64"], base["g64"]) and np.array_equal(same["out64"], base["out64"])
+    # swap one selected channel for an unselected one at each site
+    def swapped(sel, C):
+        rest = [j for j in range(C) if j not in set(int(v) for v in sel)]
+        return np.array(sorted(list(sel[1:]) + [rest[0]]), dtype=np.int32)
+    s13, s2 = swapped(base["site13"]["sel"], 32), swapped(base["site2"]["sel"], 16)
+    f13 = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, forced_sel13=s13)
+    want13 = M._force_selection(x, base["site13"], s13)
+    assert np.array_equal(f13["site13"]["r_codes"], want13["r_codes"]) and np.array_equal(f13["site13"]["sel"], s13)
+    xt = R.reconstruct_real(want13)
+    for row in range(18):
+        t = int(base["perm"][row]) // 2
+        e = int(base["ids"].reshape(-1)[base["perm"][row]])
+        w13e = _scalar_dequant(w13["codes"][e], w13["sf"][e], w13["gs"][e])
+        assert np.allclose(f13["g64"][row], _triple_loop([xt[t].tolist()], w13e.tolist())[0], rtol=1e-12, atol=1e-15)
+    assert not np.array_equal(f13["g64"], base["g64"])
+    # site 2, on an overriding h as the staged comparison uses it
+    f2 = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, h_override=base["h"], forced_sel2=s2)
+    want2 = M._force_selection(base["h"], base["site2"], s2)
+    assert np.array_equal(f2["site2"]["r_codes"], want2["r_codes"])
+    assert np.allclose(f2["out64"], _second_half_by_loops(f2, R.reconstruct_real(want2), w2), rtol=1e-11, atol=1e-14)
+    assert not np.array_equal(f2["out64"], base["out64"])
+
+
+def test_residual_scale_readings_agree_on_the_benchmark_distributions():
+    """The residual is quantized with its activation's per-tensor scale (the
+    reading taken) or with its own amax-derived one (the other reading of Eq.
+    residual-recon).  On activations drawn like the large MoE workload the two
+    correct the same amount, and the shared scale leaves the residual's block
+    scales in E4M3's normal range; only with an outlier beyond a few thousand
+    times the typical block maximum do they start to fall into the subnormals."""
+    sh = synth.MOE_SHAPES["large"]
+    x, _ = synth.activations(sh)
+    x = x[:96].to(torch.float32).numpy()
+    K = x.shape[1]
+    base = R.rac(x, 0)
+    e0 = np.linalg.norm(Q.dequantize_real(base["codes"], base["sf"], base["gs"]) - x)
+    for pct in (12.5, 50.0, 100.0):
+        n = int(K * pct / 100)
+        shared, own = R.rac(x, n), R.rac(x, n, None, "own")
+        es = np.linalg.norm(R.reconstruct_real(shared) - x) / e0
+        eo = np.linalg.norm(R.reconstruct_real(own) - x) / e0
+        assert abs(es - eo) < 5e-3 * eo, (pct, es, eo)
+        assert own["r_gs"] < shared["r_gs"] / 6                  # the residual is at least a grid step below
+    full = R.rac(x, K)
+    sub = ((full["r_sf"] > 0) & (full["r_sf"] < 8)).mean()      # E4M3 codes 1..7 are subnormal
+    assert sub < 1e-3 and (full["r_sf"] == 0).mean() < 1e-3
+    # one extreme outlier (3e4 against block maxima near 2.5) pushes the shared-scale residual scales into
+    # the subnormal codes, where the own-scale reading keeps correcting
+    y = x.copy()
+    y[0, 0] = 30000.0
+    fs, fo = R.rac(y, K), R.rac(y, K, None, "own")
+    assert ((fs["r_sf"] > 0) & (fs["r_sf"] < 8)).mean() > 0.5
+    assert ((fo["r_sf"] > 0) & (fo["r_sf"] < 8)).mean() < 0.05
+    by = R.rac(y, 0)
+    e0y = np.linalg.norm(Q.dequantize_real(by["codes"], by["sf"], by["gs"]) - y)
+    assert np.linalg.norm(R.reconstruct_real(fo) - y) < np.linalg.norm(R.reconstruct_real(fs) - y) < e0y

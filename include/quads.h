@@ -290,6 +290,28 @@ quads_status quads_moe_set_stage_trace(int32_t enable);
 int32_t quads_moe_get_stage_trace(const char** names /* host */, float* ms /* host */, int32_t cap);
 
 /*
+ * Measurement aid (no counterpart in the paper): the tensor-pipe probe.  One
+ * persistent CTA per SM keeps one pipeline stage of FP4 operands and UE4M3 scale
+ * atoms (the grouped GEMM's stage layout, quads_fp4_pipe_probe_operand_bytes()
+ * bytes copied once from `operands`, device memory, 16-byte aligned) resident in
+ * shared memory and issues `k_steps` times what the GEMM's main loop issues per
+ * K = 64 step, with no global traffic in the loop:
+ *   mode 0  one 128 x 256 x 64 block-scaled MMA per step (the bare pipe);
+ *   mode 1  two MMAs + four scale copies per step (first projection with RAC);
+ *   mode 2  one MMA + three scale copies (plain W4A4);
+ *   mode 3  two MMAs, no copies;  mode 4  as mode 1 with the copies issued by a
+ *   second thread.
+ * Time it with events on `cuda_stream`; *flop_out (host, may be NULL) receives
+ * the floating-point operations of the launch (2 * 128 * 256 * 64 per MMA and
+ * SM).  Scale bytes in `operands` should avoid the NaN code 0x7F.  The wait for
+ * the pipe to drain is bounded; a give-up writes QUADS_ERR_TIMEOUT to
+ * *status_word (device int32, zero it first).
+ */
+quads_status quads_fp4_pipe_probe(int32_t mode, int32_t k_steps, const void* operands, size_t operand_bytes,
+                                  int32_t* status_word, double* flop_out /* host */, void* cuda_stream);
+size_t quads_fp4_pipe_probe_operand_bytes(void);
+
+/*
  * Test hook (no counterpart in the paper): exercises the give-up path of a
  * bounded device-side wait without faulting or hanging anything.  It sets the
  * bound, in SM clock cycles, of the wait in which the CTAs of

@@ -302,3 +302,17 @@ def moe_get_stage_trace():
     ms = (C.c_float * 40)()
     n = lib.quads_moe_get_stage_trace(names, ms, 40)
     return [(names[i].decode(), ms[i]) for i in range(n)]
+
+
+lib.quads_fp4_pipe_probe.restype = _i32
+lib.quads_fp4_pipe_probe.argtypes = [_i32, _i32, _p, _sz, _p, C.POINTER(C.c_double), _p]
+lib.quads_fp4_pipe_probe_operand_bytes.restype = _sz
+lib.quads_fp4_pipe_probe_operand_bytes.argtypes = []
+
+
+def fp4_pipe_probe(mode, k_steps, operands, status_word):
+    """Enqueue the tensor-pipe probe; returns the floating-point operations of the launch."""
+    flop = C.c_double()
+    check(lib.quads_fp4_pipe_probe(mode, k_steps, _ptr(operands), operands.numel() * operands.element_size(),
+                                   _ptr(status_word), C.byref(flop), _stream()))
+    return flop.value

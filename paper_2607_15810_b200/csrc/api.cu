@@ -679,14 +679,17 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   // The dispatched copies of Q(x) need only the dispatch order and the codes: with a side stream
   // they are written there, next to the channel selection; the residual copies (which need the
   // selection) follow on the main stream.
-  const int64_t scatter_chunks = (int64_t)T * (H / 32);
-  const unsigned scatter_grid = (unsigned)((scatter_chunks + 255) / 256);
   const bool split_scatter = side != nullptr && nsel13 > 0;
+  auto dispatch = [&](int parts, cudaStream_t s_) {
+    return launch_kernel(rac_dispatch_kernel, dim3(L.m_tiles_max), dim3(256), (size_t)(0), s_, H, parts, mask13, header,
+                         tile_rows, row_token, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad),
+                         P(L.xsf), P(L.rq_pad), P(L.rsf));
+  };
   if (side) {
     if (split_scatter) {
       QUADS_CUDA_OK(cudaEventRecord(side->mid, st));
       QUADS_CUDA_OK(cudaStreamWaitEvent(side->stream, side->mid, 0));
-      QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3(scatter_grid), dim3(256), (size_t)(0), side->stream, T, H, 1, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
+      QUADS_CUDA_OK(dispatch(1, side->stream));
     }
   }
   if (nsel13 > 0) {
@@ -702,7 +705,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   {
     const int parts = split_scatter ? 2 : (nsel13 > 0 ? 3 : 1);
-    QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3(scatter_grid), dim3(256), (size_t)(0), st, T, H, parts, mask13, topk, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
+    QUADS_CUDA_OK(dispatch(parts, st));
+    if (nsel13 > 0 && (a->rq || a->rsf)) {
+      // verification export of the masked residual in token order (no dispatched copies: top-k of 0)
+      const int64_t chunks = (int64_t)T * (H / 32);
+      QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3((unsigned)((chunks + 255) / 256)), dim3(256), (size_t)(0), st, T, H, 2, mask13, 0, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
+    }
   }
   trace_mark("rac_dispatch", st);
   // ---- tensor maps

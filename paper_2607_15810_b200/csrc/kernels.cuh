@@ -48,6 +48,10 @@ __global__ void rac_scatter_kernel(int T, int H, int parts, const uint8_t* mask,
                                    const int32_t* pos_pad, const uint8_t* xq, const uint8_t* xsf, const uint8_t* rq,
                                    const uint8_t* rsf, uint8_t* xq_pad, uint8_t* xsf_tiled, uint8_t* rq_pad,
                                    uint8_t* rsf_tiled, uint8_t* rq_exp, uint8_t* rsf_exp);
+__global__ void rac_dispatch_kernel(int H, int parts, const uint8_t* mask, const int32_t* header,
+                                    const int32_t* tile_rows, const int32_t* row_token, const uint8_t* xq,
+                                    const uint8_t* xsf, const uint8_t* rq, const uint8_t* rsf, uint8_t* xq_pad,
+                                    uint8_t* xsf_tiled, uint8_t* rq_pad, uint8_t* rsf_tiled);
 __global__ void mask_codes_kernel(uint8_t* codes, const int* n_rows_ptr, int C, const uint8_t* mask);
 __global__ void combine_kernel(const uint16_t* y_pad, const int32_t* pos_pad, const float* wts, int T, int H,
                                int topk, uint16_t* out);

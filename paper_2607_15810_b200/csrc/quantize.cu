@@ -910,6 +910,118 @@ rac_scatter_kernel(int T, int H, int parts, const uint8_t* __restrict__ mask, in
   }
 }
 
+// ---------------------------------------------------------------------------
+// Site-13 dispatch, driven by the DESTINATION: one CTA per 128-row tile of the padded dispatch
+// order gathers its rows' codes and scales from the token-order arrays (which stay in L2: every
+// token row is read top-k times) and writes the tile's 128 x H/2 code bytes and its scale atoms
+// as whole, contiguous regions.  Written from the source side instead (one thread per token
+// chunk), every 512-byte scale atom is touched by 128 different tokens at 128 different times,
+// 4 bytes each: partially written sectors get evicted and the memory system pays for them.
+// The residual is masked (Eq. residual-recon) and sign-flipped on the way, as above.
+// grid = upper bound of the tile count (tiles beyond header[kHdrMTiles] leave at once), 256 threads.
+// ---------------------------------------------------------------------------
+constexpr int kDispatchSlab = 32;                   // scale atoms (K = 64 each) staged per pass
+__global__ void __launch_bounds__(256)
+rac_dispatch_kernel(int H, int parts, const uint8_t* __restrict__ mask, const int32_t* __restrict__ header,
+                    const int32_t* __restrict__ tile_rows, const int32_t* __restrict__ row_token,
+                    const uint8_t* __restrict__ xq, const uint8_t* __restrict__ xsf, const uint8_t* __restrict__ rq,
+                    const uint8_t* __restrict__ rsf, uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled,
+                    uint8_t* __restrict__ rq_pad, uint8_t* __restrict__ rsf_tiled) {
+  pdl_sync();
+  const int mt = blockIdx.x;
+  if (mt >= header[kHdrMTiles]) return;
+  const int n_rows = tile_rows[mt];
+  __shared__ int tok[128];
+  __shared__ __align__(16) uint8_t atoms[2][kDispatchSlab * 512];
+  if (threadIdx.x < 128) tok[threadIdx.x] = threadIdx.x < n_rows ? row_token[mt * 128 + threadIdx.x] : -1;
+  __syncthreads();
+  const bool do_x = (parts & 1) != 0, do_r = (parts & 2) != 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int per_row = H >> 5;                         // 16-byte chunks of codes per row
+  const size_t row_bytes = (size_t)(H >> 1);
+  // ---- codes: a warp walks rows warp, warp + 8, ...; its lanes take consecutive 16-byte chunks
+  for (int c = lane; c < per_row; c += 32) {
+    uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;
+    if (do_r) {
+      const uint8_t* m = mask + c * 32;
+      m0 = nibble_mask8(m); m1 = nibble_mask8(m + 8); m2 = nibble_mask8(m + 16); m3 = nibble_mask8(m + 24);
+    }
+    for (int r0 = warp; r0 < n_rows; r0 += 32) {      // four rows in flight per thread
+      uint4 xv[4], rv[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = r0 + 8 * j;
+        if (r < n_rows) {
+          const size_t so = (size_t)tok[r] * row_bytes + (size_t)c * 16;
+          if (do_x) xv[j] = __ldg(reinterpret_cast<const uint4*>(xq + so));
+          if (do_r) rv[j] = __ldg(reinterpret_cast<const uint4*>(rq + so));
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = r0 + 8 * j;
+        if (r < n_rows) {
+          const size_t po = (size_t)(mt * 128 + r) * row_bytes + (size_t)c * 16;
+          if (do_x) __stcs(reinterpret_cast<uint4*>(xq_pad + po), xv[j]);
+          if (do_r) {
+            uint4 v = rv[j];
+            v.x = (v.x & m0) ^ 0x88888888u; v.y = (v.y & m1) ^ 0x88888888u;
+            v.z = (v.z & m2) ^ 0x88888888u; v.w = (v.w & m3) ^ 0x88888888u;
+            __stcs(reinterpret_cast<uint4*>(rq_pad + po), v);
+          }
+        }
+      }
+    }
+  }
+  // ---- scales: the rows' linear scale bytes are transposed into whole atoms through shared memory
+  const int kt_count = H >> 6;
+  const size_t sf_row = (size_t)(H >> 4);
+  for (int k0 = 0; k0 < kt_count; k0 += kDispatchSlab) {
+    const int nk = min(kDispatchSlab, kt_count - k0);
+    __syncthreads();                                  // the previous slab has been written out
+    for (int i = threadIdx.x; i < nk * 32; i += blockDim.x) {
+      if (do_x) reinterpret_cast<uint4*>(atoms[0])[i] = make_uint4(0, 0, 0, 0);
+      if (do_r) reinterpret_cast<uint4*>(atoms[1])[i] = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    // a thread moves 16 bytes = four atoms' worth of one row; consecutive threads take consecutive pieces
+    const int pieces = (nk + 3) >> 2;
+    for (int i = threadIdx.x; i < n_rows * pieces; i += blockDim.x) {
+      const int r = i / pieces, pc = i - r * pieces;
+      const size_t so = (size_t)tok[r] * sf_row + (size_t)(k0 + 4 * pc) * 4;
+      const int dst = (r & 31) * 16 + (r >> 5) * 4;
+      const int n4 = min(4, nk - 4 * pc);
+      const bool wide = n4 == 4 && (sf_row & 15) == 0;   // else: word loads (row tails, rows that are not 16-byte aligned)
+      if (do_x) {
+        uint32_t w[4] = {0, 0, 0, 0};
+        if (wide) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(xsf + so));
+          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else {
+          for (int j = 0; j < n4; ++j) w[j] = __ldg(reinterpret_cast<const uint32_t*>(xsf + so) + j);
+        }
+        for (int j = 0; j < n4; ++j) *reinterpret_cast<uint32_t*>(&atoms[0][(4 * pc + j) * 512 + dst]) = w[j];
+      }
+      if (do_r) {
+        uint32_t w[4] = {0, 0, 0, 0};
+        if (wide) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(rsf + so));
+          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else {
+          for (int j = 0; j < n4; ++j) w[j] = __ldg(reinterpret_cast<const uint32_t*>(rsf + so) + j);
+        }
+        for (int j = 0; j < n4; ++j) *reinterpret_cast<uint32_t*>(&atoms[1][(4 * pc + j) * 512 + dst]) = w[j];
+      }
+    }
+    __syncthreads();
+    const size_t ao = ((size_t)mt * kt_count + k0) * 512u;
+    for (int i = threadIdx.x; i < nk * 32; i += blockDim.x) {
+      if (do_x) __stcs(reinterpret_cast<uint4*>(xsf_tiled + ao) + i, reinterpret_cast<const uint4*>(atoms[0])[i]);
+      if (do_r) __stcs(reinterpret_cast<uint4*>(rsf_tiled + ao) + i, reinterpret_cast<const uint4*>(atoms[1])[i]);
+    }
+  }
+}
+
 // Clear (in place) the codes of unselected channels of a padded [rows, C/2]
 // code matrix; one thread per 16 bytes (32 channels).  A thread keeps its column
 // chunk (its four nibble-mask words are formed once) and walks down the rows.

@@ -203,6 +203,60 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def kernel_source_digest():
+    """SHA-256 over the sources of the grouped GEMM (what an ncu capture of it depends on)."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("gemm.cu", "tcgen05.cuh", "kernels.cuh", "common.cuh"):
+        with open(os.path.join(ROOT, "paper_2607_15810_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(summary_name):
+    """(bytes per launch, note) from the `traffic_bytes_per_launch:` / `kernel_source_digest:` lines of an
+    ncu summary under profiles/; (None, why) when the summary is missing or was taken on other sources."""
+    path = os.path.join(ROOT, "profiles", summary_name)
+    try:
+        with open(path) as fh:
+            text = fh.read()
+    except OSError:
+        return None, "no ncu summary"
+    vals = {}
+    for ln in text.splitlines():
+        for key in ("traffic_bytes_per_launch", "kernel_source_digest"):
+            if ln.strip().startswith(key + ":"):
+                vals[key] = ln.split(":", 1)[1].strip()
+    if "traffic_bytes_per_launch" not in vals:
+        return None, "summary has no traffic line"
+    if vals.get("kernel_source_digest") != kernel_source_digest():
+        return None, "ncu summary predates the current kernel sources (digest %s, now %s)" % (
+            vals.get("kernel_source_digest"), kernel_source_digest())
+    return int(vals["traffic_bytes_per_launch"]), "profiles/" + summary_name
+
+
+def pipe_probe(B, torch, dev):
+    """Measured dense-FP4 rate of the tensor pipe: the library's probe kernel (operands resident in shared
+    memory, no global traffic), about 20 ms per mode so that clocks settle under the power cap."""
+    n = B.lib.quads_fp4_pipe_probe_operand_bytes()
+    g = torch.Generator(device=dev).manual_seed(1)
+    ops = torch.randint(0, 256, (n,), dtype=torch.uint8, device=dev, generator=g)
+    ops[4 * 16384:] = torch.randint(0x30, 0x40, (n - 4 * 16384,), dtype=torch.uint8, device=dev, generator=g)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    out = {}
+    for mode, name, steps in ((0, "mma_only", 200000), (1, "rac_mix_2mma_4copies", 100000), (2, "plain_mix_1mma_3copies", 200000)):
+        B.fp4_pipe_probe(mode, 2000, ops, st)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        flop = B.fp4_pipe_probe(mode, steps, ops, st)
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = flop / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    assert st.item() == 0, "the probe's bounded wait gave up"
+    return out
+
+
 def run_fake_quant_only(args):
     """16 experts' W13 of the AQAT workload through quads_fake_quant_weights: 403 MB in, 516 MB out."""
     import torch
@@ -408,10 +462,10 @@ def run_ours(args):
                 "traffic": None, "ms": g1_ms,
                 "gemm2": {"ms": g2_ms, "achieved": f_alg2 / (g2_ms * 1e-3) / 1e12, "frac": f_alg2 / (g2_ms * 1e-3) / 1e12 / fp4_peak},
                 "frac_of_nominal_9pf": ach / 9000.0}
-    # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM-1 launch, from the ncu capture
-    # summarised in profiles/gemm_kernel_moe_prefill_ncu_full.md (prefill workload, RAC at both sites)
+    # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM-1 launch: taken from the ncu summary of this
+    # workload, and only while the kernel's sources still are the ones that capture ran (else null)
     if args.workload == "prefill" and args.variant == "both":
-        roofline["traffic"] = 463474432
+        roofline["traffic"], roofline["traffic_source"] = ncu_traffic("gemm_kernel_moe_prefill_ncu_full.md")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp4 (e2m1 x e2m1, ue4m3 block scales, fp32 accumulate)",
@@ -429,6 +483,14 @@ def run_ours(args):
 
     if not args.no_aux:
         aux = {}
+        # measured dense-FP4 rate of the tensor pipe (block-scaled tcgen05.mma issue loop, no global traffic)
+        probe = pipe_probe(B, torch, dev)
+        aux["fp4_pipe_peak_tflops"] = probe["mma_only"]
+        aux["fp4_pipe_probe_tflops"] = probe
+        aux["fp4_pipe_note"] = ("executed TFLOP/s of 128x256x64 block-scaled MMAs issued from shared memory by one thread per SM, "
+                                "~20 ms per mode under the power cap; the RAC mix executes 4/3 of its algorithmic flops")
+        roofline["measured_pipe_peak"] = probe["mma_only"]
+        roofline["frac_of_measured_pipe_peak"] = ach / probe["mma_only"]
         # quantize GB/s on the activation tensor of this workload (ring of 8 inputs > L2)
         ring = [torch.randn(T, H, device=dev).to(torch.bfloat16) for _ in range(8)]
         q = torch.empty(T, H // 2, dtype=torch.uint8, device=dev)

@@ -197,7 +197,9 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
  * requantized with `a2_gs`, out = sum_k weight_k * W2 h~.
  *
  * Dense mode (I == 0): one projection out[T, N] = W X~ with E = topk = 1, the
- * weight in w13_*, no routing, no SwiGLU ("single dense W4A4+RAC GEMM").
+ * weight in w13_*, no routing, no SwiGLU ("single dense W4A4+RAC GEMM").  With
+ * operand_mode = QUADS_W4A16 / QUADS_W16A4 the same projection is computed with
+ * only the weights / only the activations in NVFP4 (see the enum below).
  *
  * Weight buffers are exactly what quads_fake_quant_weights() writes with
  * QUADS_SF_TILED: w13 is [E, 2I, H] (gate rows first, then up rows), w2 is
@@ -220,6 +222,15 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
  * would enqueue into the capturing side stream).  The timing and trace aids
  * below keep process-wide state and are not thread-safe.
  */
+enum {
+  QUADS_W4A4 = 0,   /* both operands NVFP4, block-scaled FP4 tensor-core product (+ RAC) */
+  QUADS_W4A16 = 1,  /* NVFP4 weights (w13_q / w13_sf / w13_gs) decoded to bf16, x stays bf16: out = bf16(W^) x,
+                       a bf16 tensor-core product with float32 accumulation -- also the learner's forward of
+                       Eq. "w4a16-qat-forward" */
+  QUADS_W16A4 = 2   /* x quantized online (a13_gs or amax-derived) and decoded to bf16, weights bf16 (w13_bf16):
+                       out = W bf16(Q_A(x)) */
+};
+
 typedef struct {
   int32_t T, H, I, E, topk;
   int32_t N;                    /* dense mode only */
@@ -257,6 +268,11 @@ typedef struct {
   int32_t* sel2;                /* [rac_nsel_2] ascending */
   void* workspace;
   size_t workspace_bytes;       /* >= quads_moe_workspace_bytes(T, H, I, E, topk, N) */
+  /* Dense mode only: which operands are NVFP4 (the one-sided rollout modes of Table
+     "qdq-alignment" and Section "Train-inference mismatch ...").  Modes 1 and 2 take no RAC
+     (rac_nsel_13 must be 0): they exist to isolate one side's quantization error. */
+  int32_t operand_mode;         /* QUADS_W4A4 (0, default), QUADS_W4A16 or QUADS_W16A4 */
+  const void* w13_bf16;         /* QUADS_W16A4: the unquantized weight, bf16 [N, H], 16-byte aligned */
 } quads_moe_args;
 
 quads_status quads_moe_w4a4_rac(const quads_moe_args* args /* host */, void* cuda_stream);

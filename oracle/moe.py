@@ -81,6 +81,29 @@ def dense_w4a4_rac(x, w_codes, w_sf, w_gs, n_sel, a_gs=None, r_gs=None):
     return dict(site=site, y64=y64, y=F.bf16_round(y64), absdot=absdot)
 
 
+def dense_w4a16(x, w_codes, w_sf, w_gs):
+    """One-sided mode "W4A16" (Table "qdq-alignment"; also the learner's forward of Eq.
+    w4a16-qat-forward): Y = W^ X with W^ = QDQ_W(W) as the bf16 tensor the trainer multiplies
+    by, activations left in bf16.  x float32 (bf16-valued) [T, K].  The contraction is the
+    plain definition in float64.  Returns dict(y64, y, absdot)."""
+    w = Q.dequantize_bf16(w_codes, w_sf, w_gs).astype(np.float64)
+    x64 = np.asarray(x, dtype=np.float64)
+    y64 = x64 @ w.T
+    return dict(y64=y64, y=F.bf16_round(y64), absdot=np.abs(x64) @ np.abs(w).T)
+
+
+def dense_w16a4(x, w_bf16, a_gs=None):
+    """One-sided mode "W16A4": Y = W QDQ_A(X), activations quantized as the rollout does (Eq.
+    act-error-def) and decoded to bf16, weights left in bf16 ([N, K] float32, bf16-valued).
+    Returns dict(codes, sf, gs of the activation, y64, y, absdot)."""
+    x = np.asarray(x, dtype=F32)
+    codes, sf8, gs = Q.quantize(x, a_gs)
+    xh = Q.dequantize_bf16(codes, sf8, gs).astype(np.float64)
+    w64 = np.asarray(w_bf16, dtype=np.float64)
+    y64 = xh @ w64.T
+    return dict(codes=codes, sf=sf8, gs=gs, y64=y64, y=F.bf16_round(y64), absdot=np.abs(xh) @ np.abs(w64).T)
+
+
 def _absdot(site, w_abs):
     """sum_k |a_k * b_k| over every product the tensor cores form: the main
     term and the residual term (the tolerance of the GEMM comparison scales

@@ -33,6 +33,7 @@ class MoEArgs(C.Structure):
         ("xq", _p), ("xsf", _p), ("rq", _p), ("rsf", _p), ("sel13", _p), ("a13_gs_out", _p),
         ("h_bf16", _p), ("hq", _p), ("hsf", _p), ("r2q", _p), ("r2sf", _p), ("sel2", _p),
         ("workspace", _p), ("workspace_bytes", _sz),
+        ("operand_mode", _i32), ("w13_bf16", _p),
     ]
 
 
@@ -264,6 +265,39 @@ def dense_w4a4_rac(x, w, nsel, a_gs=None, export=False, workspace=None):
         res["a13_gs"] = torch.empty(1, dtype=torch.float32, device=dev)
         a.xq, a.xsf, a.rq, a.rsf = map(_ptr, (res["xq"], res["xsf"], res["rq"], res["rsf"]))
         a.sel13, a.a13_gs_out = _ptr(res["sel13"]), _ptr(res["a13_gs"])
+    ws = workspace if workspace is not None else _ws(moe_workspace_bytes(T, K, 0, 1, 1, N), dev)
+    a.workspace, a.workspace_bytes = _ptr(ws), ws.numel()
+    check(lib.quads_moe_w4a4_rac(C.byref(a), _stream()))
+    res["workspace"] = ws
+    return res
+
+
+W4A4, W4A16, W16A4 = 0, 1, 2
+
+
+def dense_one_sided(x, mode, w=None, w_bf16=None, a_gs=None, export=False, workspace=None):
+    """The one-sided rollout modes of the dense projection: mode = W4A16 (w: packed NVFP4 weight
+    dict, x stays bf16) or W16A4 (w_bf16: bf16 [N, K] weight, x quantized online and decoded).
+    Returns dict(out=bf16 [T, N], ...)."""
+    T, K = x.shape
+    N = w["q"].shape[-2] if mode == W4A16 else w_bf16.shape[0]
+    dev = x.device
+    a = MoEArgs()
+    a.T, a.H, a.I, a.E, a.topk, a.N = T, K, 0, 1, 1, N
+    a.x = _ptr(x)
+    a.operand_mode = mode
+    if mode == W4A16:
+        a.w13_q, a.w13_sf, a.w13_gs = _ptr(w["q"]), _ptr(w["sf"]), _ptr(w["gs"])
+    else:
+        a.w13_bf16 = _ptr(w_bf16)
+        a.a13_gs = _ptr(a_gs)
+    res = {"out": torch.empty(T, N, dtype=torch.bfloat16, device=dev)}
+    a.out = _ptr(res["out"])
+    if export and mode == W16A4:
+        res["xq"] = torch.empty(T, K // 2, dtype=torch.uint8, device=dev)
+        res["xsf"] = torch.empty(T, K // 16, dtype=torch.uint8, device=dev)
+        res["a13_gs"] = torch.empty(1, dtype=torch.float32, device=dev)
+        a.xq, a.xsf, a.a13_gs_out = _ptr(res["xq"]), _ptr(res["xsf"]), _ptr(res["a13_gs"])
     ws = workspace if workspace is not None else _ws(moe_workspace_bytes(T, K, 0, 1, 1, N), dev)
     a.workspace, a.workspace_bytes = _ptr(ws), ws.numel()
     check(lib.quads_moe_w4a4_rac(C.byref(a), _stream()))

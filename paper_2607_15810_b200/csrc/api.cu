@@ -94,6 +94,22 @@ quads_status make_sf_map(CUtensorMap* map, const void* base, uint64_t atoms) {
   return r == CUDA_SUCCESS ? QUADS_OK : QUADS_ERR_CUDA;
 }
 
+// 2D map over a bf16 matrix [rows, K] (K contiguous): box 64 elements (128 bytes) x 128 rows,
+// 128-byte swizzle, zero fill outside.
+quads_status make_bf16_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t K) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return QUADS_ERR_CUDA;
+  if (rows == 0) rows = 1;
+  cuuint64_t dims[2] = {K, rows};
+  cuuint64_t strides[1] = {K * 2};
+  cuuint32_t box[2] = {64, 128};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? QUADS_OK : QUADS_ERR_CUDA;
+}
+
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // ------------------------------------------------------------------ workspace
@@ -101,7 +117,7 @@ struct MoeLayout {
   size_t header, amax, counters13, counters2, expert_total, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
   size_t perm, pos_pad, row_token, row_weight;
   size_t partials13, scores13, keys13, keys2, sel13, mask13, xq_tok, xsf_tok, rq_tok, rsf_tok, xq_pad, xsf, rq_pad, rsf;
-  size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad;
+  size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad, dec;
   size_t total;
   int n_chunks, m_tiles_max, stats_ctas, rows_per_cta;
 };
@@ -164,7 +180,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
     L.mask2 = take((size_t)I);
     L.y_pad = take(pad_rows * (size_t)H * 2);
   }
-  (void)N;
+  if (dense) L.dec = take((size_t)std::max(T, N) * (size_t)H * 2);   // decoded bf16 operand of the one-sided modes
   L.total = o;
   return L;
 }
@@ -553,8 +569,17 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   if (H > 16384 || I > 16384 || a->rac_nsel_13 < 0 || a->rac_nsel_13 > H || (!dense && (a->rac_nsel_2 < 0 || a->rac_nsel_2 > I)))
     return QUADS_ERR_SHAPE;
   if ((int64_t)T * topk > 0x3FFFFFFF) return QUADS_ERR_SHAPE;
+  if (a->operand_mode != QUADS_W4A4) {
+    if (!dense || (a->operand_mode != QUADS_W4A16 && a->operand_mode != QUADS_W16A4) || a->rac_nsel_13 != 0)
+      return QUADS_ERR_SHAPE;
+  }
   if (T == 0) return QUADS_OK;                      // nothing to do; x / out may be NULL
-  if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) return QUADS_ERR_NULL;
+  if (a->operand_mode == QUADS_W16A4) {
+    if (!a->x || !a->w13_bf16 || !a->out) return QUADS_ERR_NULL;
+    if (!aligned(a->w13_bf16, 16)) return QUADS_ERR_SHAPE;
+  } else if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) {
+    return QUADS_ERR_NULL;
+  }
   if (!dense && (!a->router_logits || !a->w2_q || !a->w2_sf || !a->w2_gs || !a->a2_gs)) return QUADS_ERR_NULL;
   if (!aligned(a->x, 32) || !aligned(a->w13_q, 16) || !aligned(a->w13_sf, 16) || !aligned(a->out, 16) ||
       (!dense && (!aligned(a->w2_q, 16) || !aligned(a->w2_sf, 16))))
@@ -590,6 +615,34 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   // header (status word included) and the amax word start at zero
   QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, L.ids, st));
   trace_mark("memset", st);
+
+  if (dense && a->operand_mode != QUADS_W4A4) {
+    // ---- one-sided modes: decode the NVFP4 side to bf16 with the library's own kernels, then one
+    // bf16 tensor-core product
+    uint16_t* dec = reinterpret_cast<uint16_t*>(P(L.dec));
+    const void *A_op = a->x, *B_op = a->w13_bf16;
+    if (a->operand_mode == QUADS_W4A16) {
+      const int64_t nblk = (int64_t)a->N * (H / 16);
+      const int grid = (int)std::min<int64_t>((nblk + 255) / 256, (int64_t)di.sm_count * 16);
+      QUADS_CUDA_OK(launch_kernel(dequantize_kernel, dim3(grid), dim3(256), (size_t)0, st, a->w13_q, a->w13_sf, a->w13_gs, 1,
+                                  nblk, (uint32_t)(H / 16), (int)(H / 64), 1, (int64_t)quads_sf_tiled_bytes(a->N, H), dec));
+      B_op = dec;
+    } else {
+      // Q_A(x) then decode, in one pass of the quantizer (its scratch: the 256 bytes at the amax slot)
+      const int launches = g_launch_count;
+      s = quantize_common(a->x, 1, T, H, H, 0, a->a13_gs, dec, a->xq, a->xsf, a->a13_gs_out, QUADS_SF_LINEAR, P(L.amax), 256, st);
+      g_launch_count += launches;
+      if (s != QUADS_OK) return s;
+      A_op = dec;
+    }
+    CUtensorMap tm_a, tm_b;
+    if ((s = make_bf16_map(&tm_a, A_op, (uint64_t)T, (uint64_t)H)) != QUADS_OK) return s;
+    if ((s = make_bf16_map(&tm_b, B_op, (uint64_t)a->N, (uint64_t)H)) != QUADS_OK) return s;
+    s = launch_gemm_bf16(tm_a, tm_b, T, a->N, H, static_cast<uint16_t*>(a->out), header + kHdrStatus, di.sm_count, st);
+    if (s != QUADS_OK) return s;
+    QUADS_CUDA_OK(cudaGetLastError());
+    return QUADS_OK;
+  }
 
   // ---- routing and dispatch order: on a side stream, next to the activation chain below
   // (declared in this order: on an early return the guard joins first, then the lock is released)

@@ -130,6 +130,11 @@ struct GemmMaps {
 bool gemm_swapped_ok(int64_t assignments, int n_experts, int m_tiles_max);
 quads_status launch_gemm_swapped(int epi, const GemmParams& p, const GemmMaps& m, int n_sms, cudaStream_t stream);
 
+// ---- gemm_bf16.cu: out[T, N] = A[T, K] B[N, K]^T, bf16 operands (tensor maps with boxes of 64 x 128
+// elements, 128-byte swizzle), float32 accumulation, bf16 output; K % 64 == 0, N % 128 == 0
+quads_status launch_gemm_bf16(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int T, int N, int K, uint16_t* out,
+                              int32_t* status, int n_sms, cudaStream_t stream);
+
 quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const GemmMaps& m, int n_sms,
                          cudaStream_t stream);
 

@@ -452,3 +452,41 @@ def test_compensating_more_channels_shrinks_the_mismatch_against_the_learner(B):
     assert all(a > b for a, b in zip(errs, errs[1:])), errs
     assert errs[-1] < 0.25 * errs[0], errs
     assert 0.01 < errs[0] < 0.3, errs            # plain W4A4: a few per cent, as NVFP4 activations give
+
+
+@pytest.mark.parametrize("T,K,N,seed", [(128, 512, 256, 0), (300, 2048, 384, 6), (1, 128, 128, 1), (2300, 1024, 640, 9)])
+def test_one_sided_modes_of_the_dense_projection(B, T, K, N, seed):
+    """W4A16 (NVFP4 weights decoded to bf16, activations untouched) and W16A4 (activations through Q_A and
+    back, bf16 weights): the ablation modes of Table "qdq-alignment", bf16 tensor-core products, against
+    the float64 oracle; the quantized side's bytes are the ones the W4A4 path uses."""
+    x, w = synth.dense_inputs(seed, T=T, K=K, N=N)
+    wo = MC.oracle_weights(w[None])
+    wq = B.fake_quant_weights(w.unsqueeze(0).cuda(), want_fq=False, sf_layout=B.SF_TILED)
+    # ---- W4A16
+    res = B.dense_one_sided(x.cuda(), B.W4A16, w=wq)
+    torch.cuda.synchronize()
+    assert B.moe_async_status(res["workspace"]) == 0
+    o = M.dense_w4a16(MC.f32(x), wo["codes"][0], wo["sf"][0], wo["gs"][0])
+    got = MC.f32(res["out"]).astype(np.float64)
+    r1 = float((np.abs(got - o["y64"]) / MC.gemm_tol(o["absdot"], o["y64"])).max())
+    assert r1 <= 1.0, r1
+    # ---- W16A4, amax-derived and supplied activation scale
+    for a_gs in (None, np.float32(0.5) * Q.tensor_global_scale(MC.f32(x))):
+        gs_t = None if a_gs is None else torch.tensor([float(a_gs)]).cuda()
+        res = B.dense_one_sided(x.cuda(), B.W16A4, w_bf16=w.cuda(), a_gs=gs_t, export=True)
+        torch.cuda.synchronize()
+        assert B.moe_async_status(res["workspace"]) == 0
+        o = M.dense_w16a4(MC.f32(x), MC.f32(w), a_gs)
+        assert np.float32(res["a13_gs"].item()) == o["gs"]
+        assert np.array_equal(res["xq"].cpu().numpy(), F.pack_nibbles(o["codes"]))
+        assert np.array_equal(res["xsf"].cpu().numpy(), o["sf"])
+        got = MC.f32(res["out"]).astype(np.float64)
+        r2 = float((np.abs(got - o["y64"]) / MC.gemm_tol(o["absdot"], o["y64"])).max())
+        assert r2 <= 1.0, r2
+    # RAC is not part of these modes
+    with pytest.raises(B.QuadsError) as e:
+        a = B.MoEArgs()
+        a.T, a.H, a.I, a.E, a.topk, a.N = T, K, 0, 1, 1, N
+        a.operand_mode, a.rac_nsel_13 = B.W4A16, 16
+        B.check(B.lib.quads_moe_w4a4_rac(B.C.byref(a), None))
+    assert e.value.status == -2

@@ -401,3 +401,38 @@ def test_residual_scale_readings_agree_on_the_benchmark_distributions():
     by = R.rac(y, 0)
     e0y = np.linalg.norm(Q.dequantize_real(by["codes"], by["sf"], by["gs"]) - y)
     assert np.linalg.norm(R.reconstruct_real(fo) - y) < np.linalg.norm(R.reconstruct_real(fs) - y) < e0y
+
+
+def test_one_sided_modes_against_loops_and_their_special_cases():
+    """W4A16 / W16A4 (Table "qdq-alignment"): explicit loops on the decoded bf16 operands; an operand
+    that NVFP4 represents exactly makes its one-sided mode the plain bf16 product; and with both
+    sides exactly representable (power-of-two tensor scales, <= 6 significant bits) all of W4A4,
+    W4A16, W16A4 and the plain product coincide."""
+    x, w = synth.dense_inputs(seed=4, T=5, K=32, N=4, outlier_channels=(3,))
+    x, w = x.to(torch.float32).numpy(), w.to(torch.float32).numpy()
+    wq = _tiny_weights(1, 4, 32, 9)
+    a = M.dense_w4a16(x, wq["codes"][0], wq["sf"][0], wq["gs"][0])
+    wd = Q.dequantize_bf16(wq["codes"][0], wq["sf"][0], wq["gs"][0])
+    assert np.array_equal(F.bf16_round(wd), wd)
+    assert np.allclose(a["y64"], _triple_loop(x.tolist(), wd.astype(np.float64).tolist()), rtol=1e-12, atol=1e-15)
+    assert np.allclose(a["absdot"], _triple_loop(np.abs(x).tolist(), np.abs(wd).astype(np.float64).tolist()), rtol=1e-12)
+    b = M.dense_w16a4(x, w)
+    xq = Q.quantize(x)
+    assert np.array_equal(b["codes"], xq[0]) and np.array_equal(b["sf"], xq[1]) and b["gs"] == xq[2]
+    xd = Q.dequantize_bf16(*xq)
+    assert np.allclose(b["y64"], _triple_loop(xd.astype(np.float64).tolist(), w.astype(np.float64).tolist()), rtol=1e-12, atol=1e-15)
+    assert not np.allclose(b["y64"], x.astype(np.float64) @ w.astype(np.float64).T, rtol=1e-3)   # the activation error is there
+    # exactly representable operands: values (code) * (E4M3 scale) * 2^-p
+    mags = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6, -0.5, -1, -1.5, -2, -3, -4, -6, 6])
+    rng = np.random.default_rng(2)
+    xe = np.stack([rng.permutation(mags) * 2.0 ** rng.integers(-3, 3) for _ in range(6 * 2)]).reshape(6, 32) * 2.0 ** -4
+    we = np.stack([rng.permutation(mags) * 2.0 ** rng.integers(-3, 3) for _ in range(3 * 2)]).reshape(3, 32) * 2.0 ** -6
+    xe[0, :16] = mags * 448 * 2.0 ** -4                         # a block at the top of the range: tensor scale 2^-4
+    we[0, :16] = mags * 448 * 2.0 ** -6
+    xe, we = xe.astype(np.float32), we.astype(np.float32)
+    cw, sw, gw = Q.quantize(we)
+    assert gw == np.float32(2.0 ** -6) and np.array_equal(Q.dequantize_f32(cw, sw, gw), we)
+    plain = xe.astype(np.float64) @ we.astype(np.float64).T
+    assert np.array_equal(M.dense_w4a16(xe, cw, sw, gw)["y64"], plain)
+    assert np.array_equal(M.dense_w16a4(xe, we)["y64"], plain)
+    assert np.array_equal(M.dense_w4a4_rac(xe, cw, sw, gw, 0)["y64"], plain)

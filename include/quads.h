@@ -227,8 +227,10 @@ enum {
   QUADS_W4A16 = 1,  /* NVFP4 weights (w13_q / w13_sf / w13_gs) decoded to bf16, x stays bf16: out = bf16(W^) x,
                        a bf16 tensor-core product with float32 accumulation -- also the learner's forward of
                        Eq. "w4a16-qat-forward" */
-  QUADS_W16A4 = 2   /* x quantized online (a13_gs or amax-derived) and decoded to bf16, weights bf16 (w13_bf16):
+  QUADS_W16A4 = 2,  /* x quantized online (a13_gs or amax-derived) and decoded to bf16, weights bf16 (w13_bf16):
                        out = W bf16(Q_A(x)) */
+  QUADS_W16A16 = 3  /* neither side quantized (x and w13_bf16 in bf16): Y_train of Eq. "linear-mismatch", the
+                       reference the mismatch of the other modes is measured against */
 };
 
 typedef struct {
@@ -304,6 +306,31 @@ quads_status quads_moe_last_kernel_ms(float* gemm1_ms /* host */, float* gemm2_m
  */
 quads_status quads_moe_set_stage_trace(int32_t enable);
 int32_t quads_moe_get_stage_trace(const char** names /* host */, float* ms /* host */, int32_t cap);
+
+/*
+ * Diagnostics of the paper's mismatch analysis, computed on the device.
+ *
+ * quads_rac_channel_scores: s_j^2 = sum over the token batch of (Q_A(X) - X)[:, j]^2, the squared
+ * channel score of Eq. "channel-score" -- the per-channel residual map whose heavy channels are the
+ * "vertical bands" of Fig. "residual-distribution" and whose largest entries RAC selects.
+ *   x       bf16 [T, H], 32-byte aligned, H % 128 == 0
+ *   gs_in   float[1] per-tensor scale of x, or NULL: amax-derived on the device
+ *   scores  out, double [H] (per-CTA float32 partial sums over <= 14 rows, then float64, fixed order)
+ *   workspace >= quads_rac_channel_scores_workspace_bytes(T, H) bytes, 256-byte aligned
+ *
+ * quads_mismatch_norms: out = { ||A - B||_F^2, ||A||_F^2, ||B||_F^2 } for two bf16 tensors of n
+ * elements, float64 accumulation in a fixed order -- the layer-wise forward mismatch of Eq.
+ * "linear-mismatch" for A = Y_infer, B = Y_train (take the square root of out[0]), and, with the
+ * one-sided modes of quads_moe_w4a4_rac as A, its activation-error and weight-error terms.
+ *   a, b    bf16 [n], 16-byte aligned;  out  double [3] (device)
+ *   workspace >= quads_mismatch_norms_workspace_bytes() bytes, 256-byte aligned
+ */
+quads_status quads_rac_channel_scores(const void* x, int64_t T, int64_t H, const float* gs_in, double* scores,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+size_t quads_rac_channel_scores_workspace_bytes(int64_t T, int64_t H);
+quads_status quads_mismatch_norms(const void* a, const void* b, int64_t n, double* out, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream);
+size_t quads_mismatch_norms_workspace_bytes(void);
 
 /*
  * Measurement aid (no counterpart in the paper): the tensor-pipe probe.  One

@@ -272,7 +272,7 @@ def dense_w4a4_rac(x, w, nsel, a_gs=None, export=False, workspace=None):
     return res
 
 
-W4A4, W4A16, W16A4 = 0, 1, 2
+W4A4, W4A16, W16A4, W16A16 = 0, 1, 2, 3
 
 
 def dense_one_sided(x, mode, w=None, w_bf16=None, a_gs=None, export=False, workspace=None):
@@ -281,6 +281,7 @@ def dense_one_sided(x, mode, w=None, w_bf16=None, a_gs=None, export=False, works
     Returns dict(out=bf16 [T, N], ...)."""
     T, K = x.shape
     N = w["q"].shape[-2] if mode == W4A16 else w_bf16.shape[0]
+    assert mode in (W4A16, W16A4, W16A16)
     dev = x.device
     a = MoEArgs()
     a.T, a.H, a.I, a.E, a.topk, a.N = T, K, 0, 1, 1, N
@@ -290,7 +291,7 @@ def dense_one_sided(x, mode, w=None, w_bf16=None, a_gs=None, export=False, works
         a.w13_q, a.w13_sf, a.w13_gs = _ptr(w["q"]), _ptr(w["sf"]), _ptr(w["gs"])
     else:
         a.w13_bf16 = _ptr(w_bf16)
-        a.a13_gs = _ptr(a_gs)
+        a.a13_gs = _ptr(a_gs) if mode == W16A4 else None
     res = {"out": torch.empty(T, N, dtype=torch.bfloat16, device=dev)}
     a.out = _ptr(res["out"])
     if export and mode == W16A4:
@@ -350,3 +351,32 @@ def fp4_pipe_probe(mode, k_steps, operands, status_word):
     check(lib.quads_fp4_pipe_probe(mode, k_steps, _ptr(operands), operands.numel() * operands.element_size(),
                                    _ptr(status_word), C.byref(flop), _stream()))
     return flop.value
+
+
+lib.quads_rac_channel_scores.restype = _i32
+lib.quads_rac_channel_scores.argtypes = [_p, _i64, _i64, _p, _p, _p, _sz, _p]
+lib.quads_rac_channel_scores_workspace_bytes.restype = _sz
+lib.quads_rac_channel_scores_workspace_bytes.argtypes = [_i64, _i64]
+lib.quads_mismatch_norms.restype = _i32
+lib.quads_mismatch_norms.argtypes = [_p, _p, _i64, _p, _p, _sz, _p]
+lib.quads_mismatch_norms_workspace_bytes.restype = _sz
+lib.quads_mismatch_norms_workspace_bytes.argtypes = []
+
+
+def rac_channel_scores(x, gs=None, workspace=None):
+    """Squared channel scores of Eq. channel-score: float64 [H] (device)."""
+    T, H = x.shape
+    scores = torch.empty(H, dtype=torch.float64, device=x.device)
+    ws = workspace if workspace is not None else _ws(lib.quads_rac_channel_scores_workspace_bytes(T, H), x.device)
+    check(lib.quads_rac_channel_scores(_ptr(x), T, H, _ptr(gs), _ptr(scores), _ptr(ws), ws.numel(), _stream()))
+    return scores
+
+
+def mismatch_norms(a, b, workspace=None):
+    """float64 [3] (device): ||a - b||^2, ||a||^2, ||b||^2 over two bf16 tensors of equal size."""
+    assert a.dtype == torch.bfloat16 and b.dtype == torch.bfloat16 and a.numel() == b.numel()
+    assert a.is_contiguous() and b.is_contiguous()
+    out = torch.empty(3, dtype=torch.float64, device=a.device)
+    ws = workspace if workspace is not None else _ws(lib.quads_mismatch_norms_workspace_bytes(), a.device)
+    check(lib.quads_mismatch_norms(_ptr(a), _ptr(b), a.numel(), _ptr(out), _ptr(ws), ws.numel(), _stream()))
+    return out

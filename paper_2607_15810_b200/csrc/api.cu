@@ -501,6 +501,91 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
                          sizeof(uint32_t) * 2 * QUADS_NOALLOC_MAX_TENSORS, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---- diagnostics
+static int score_stats_ctas(int64_t T, int* rows_per_cta) {
+  int ctas = T < 592 * 4 ? (int)((T + 3) / 4) : 592;
+  if (ctas < 1) ctas = 1;
+  int rpc = (int)((T + ctas - 1) / ctas);
+  if (rpc < 1) rpc = 1;
+  ctas = (int)((T + rpc - 1) / rpc);
+  *rows_per_cta = rpc;
+  return ctas < 1 ? 1 : ctas;
+}
+
+size_t quads_rac_channel_scores_workspace_bytes(int64_t T, int64_t H) {
+  if (T < 0 || H <= 0) return 0;
+  int rpc;
+  const int ctas = score_stats_ctas(T, &rpc);
+  return 512 + align_up((size_t)((H + 31) / 32) * 4, 256) + align_up((size_t)ctas * H * 4, 256) +
+         align_up((size_t)H * 8 * kScoreSlices, 256);
+}
+
+quads_status quads_rac_channel_scores(const void* x, int64_t T, int64_t H, const float* gs_in, double* scores,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  g_launch_count = 0;
+  if (T < 0 || T > 0x3FFFFFFF || H <= 0 || (H % 128) != 0 || H > 16384) return QUADS_ERR_SHAPE;
+  if (!scores || (T > 0 && !x)) return QUADS_ERR_NULL;
+  if (!aligned(x, 32) || !aligned(scores, 8)) return QUADS_ERR_SHAPE;
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < quads_rac_channel_scores_workspace_bytes(T, H))
+    return QUADS_ERR_WORKSPACE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (T == 0) { QUADS_CUDA_OK(cudaMemsetAsync(scores, 0, (size_t)H * 8, st)); return QUADS_OK; }
+  int rpc;
+  const int ctas = score_stats_ctas(T, &rpc);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  uint32_t* amax_bits = reinterpret_cast<uint32_t*>(ws);                 // [0, 256): amax word; [256, 512): status word
+  int32_t* status_word = reinterpret_cast<int32_t*>(ws + 256);
+  unsigned int* counters = reinterpret_cast<unsigned int*>(ws + 512);
+  const size_t n_counter_bytes = align_up((size_t)((H + 31) / 32) * 4, 256);
+  float* partials = reinterpret_cast<float*>(ws + 512 + n_counter_bytes);
+  double* slices = reinterpret_cast<double*>(ws + 512 + n_counter_bytes + align_up((size_t)ctas * H * 4, 256));
+  QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, 512 + n_counter_bytes, st));
+  const uint16_t* xp = static_cast<const uint16_t*>(x);
+  if (!gs_in) {
+    const int64_t chunks = T * (H / 8);
+    int gx = (int)std::min<int64_t>((chunks + 2047) / 2048, (int64_t)di.sm_count * 8);
+    QUADS_CUDA_OK(launch_kernel(amax_kernel, dim3(gx, 1), dim3(256), (size_t)0, st, xp, T, H, H, (int64_t)0, amax_bits));
+  }
+  const int block = H / 16 > 256 ? 256 : (int)((H / 16 + 31) / 32 * 32);
+  QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(ctas), dim3(block), (size_t)0, st, xp, (int)T, (int)H, gs_in, amax_bits,
+                              (unsigned int*)nullptr, status_word, (float*)nullptr, rpc, 1, partials, (uint8_t*)nullptr,
+                              (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr));
+  // the order-preserving 64-bit keys of non-negative scores are the scores' own bit patterns
+  QUADS_CUDA_OK(launch_kernel(score_reduce_kernel, dim3((unsigned)((H + 31) / 32), kScoreSlices), dim3(256), (size_t)0, st,
+                              (const float*)partials, (const int*)nullptr, 1, ctas, (int)H, slices, counters,
+                              reinterpret_cast<unsigned long long*>(scores)));
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
+size_t quads_mismatch_norms_workspace_bytes(void) { return 256 + 1184 * 3 * sizeof(double); }
+
+quads_status quads_mismatch_norms(const void* a, const void* b, int64_t n, double* out, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
+  g_launch_count = 0;
+  if (n < 0) return QUADS_ERR_SHAPE;
+  if (!out || (n > 0 && (!a || !b))) return QUADS_ERR_NULL;
+  if (!aligned(a, 16) || !aligned(b, 16) || !aligned(out, 8)) return QUADS_ERR_SHAPE;
+  if (!workspace || !aligned(workspace, 256) || workspace_bytes < quads_mismatch_norms_workspace_bytes())
+    return QUADS_ERR_WORKSPACE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, 256, st));
+  const int64_t want = (n / 8 + 256 * 4 - 1) / (256 * 4);
+  const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(want, 1184));
+  QUADS_CUDA_OK(launch_kernel(mismatch_norms_kernel, dim3(grid), dim3(256), (size_t)0, st, static_cast<const uint16_t*>(a),
+                              static_cast<const uint16_t*>(b), n, reinterpret_cast<double*>(ws + 256),
+                              reinterpret_cast<unsigned int*>(ws), out));
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
 size_t quads_moe_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk, int32_t N) {
   if (T < 0 || H <= 0 || I < 0 || E < 1 || topk < 1) return 0;
   return moe_layout(T, H, I, E, topk, N).total;
@@ -570,11 +655,11 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     return QUADS_ERR_SHAPE;
   if ((int64_t)T * topk > 0x3FFFFFFF) return QUADS_ERR_SHAPE;
   if (a->operand_mode != QUADS_W4A4) {
-    if (!dense || (a->operand_mode != QUADS_W4A16 && a->operand_mode != QUADS_W16A4) || a->rac_nsel_13 != 0)
+    if (!dense || a->operand_mode < QUADS_W4A16 || a->operand_mode > QUADS_W16A16 || a->rac_nsel_13 != 0)
       return QUADS_ERR_SHAPE;
   }
   if (T == 0) return QUADS_OK;                      // nothing to do; x / out may be NULL
-  if (a->operand_mode == QUADS_W16A4) {
+  if (a->operand_mode == QUADS_W16A4 || a->operand_mode == QUADS_W16A16) {
     if (!a->x || !a->w13_bf16 || !a->out) return QUADS_ERR_NULL;
     if (!aligned(a->w13_bf16, 16)) return QUADS_ERR_SHAPE;
   } else if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) {
@@ -627,7 +712,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
       QUADS_CUDA_OK(launch_kernel(dequantize_kernel, dim3(grid), dim3(256), (size_t)0, st, a->w13_q, a->w13_sf, a->w13_gs, 1,
                                   nblk, (uint32_t)(H / 16), (int)(H / 64), 1, (int64_t)quads_sf_tiled_bytes(a->N, H), dec));
       B_op = dec;
-    } else {
+    } else if (a->operand_mode == QUADS_W16A4) {
       // Q_A(x) then decode, in one pass of the quantizer (its scratch: the 256 bytes at the amax slot)
       const int launches = g_launch_count;
       s = quantize_common(a->x, 1, T, H, H, 0, a->a13_gs, dec, a->xq, a->xsf, a->a13_gs_out, QUADS_SF_LINEAR, P(L.amax), 256, st);

@@ -60,6 +60,9 @@ __global__ void export_site2_kernel(int A, int I, const int32_t* perm, const int
                                     const uint8_t* r2sf_tiled, const uint8_t* mask2, uint8_t* hq, uint8_t* hsf,
                                     uint8_t* r2q, uint8_t* r2sf);
 
+__global__ void mismatch_norms_kernel(const uint16_t* a, const uint16_t* b, int64_t n, double* partials,
+                                      unsigned int* counter, double* out);
+
 // ---- routing.cu
 template <int NJ>
 __global__ void route_kernel_t(const float* logits, int T, int E, int topk, int renormalize, int32_t* ids,

@@ -720,8 +720,10 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
       unpack8(v1, f + 8);
       const BlockQ bq = quantize_block(f, qc);
       const size_t qo = (size_t)r * (H >> 1) + kb * 8, so = (size_t)r * k16 + kb;
-      *reinterpret_cast<uint2*>(xq + qo) = make_uint2(bq.lo, bq.hi);
-      xsf[so] = (uint8_t)bq.sf8;
+      if (xq) {
+        *reinterpret_cast<uint2*>(xq + qo) = make_uint2(bq.lo, bq.hi);
+        xsf[so] = (uint8_t)bq.sf8;
+      }
       if (xq_exp) *reinterpret_cast<uint2*>(xq_exp + qo) = make_uint2(bq.lo, bq.hi);
       if (xsf_exp) xsf_exp[so] = (uint8_t)bq.sf8;
       if (with_residual) {
@@ -731,9 +733,11 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
           o[i] = __fsub_rn(o[i], f[i]);
           acc[i] = __fmaf_rn(o[i], o[i], acc[i]);
         }
-        const BlockQ br = quantize_block(o, qc);
-        *reinterpret_cast<uint2*>(rq + qo) = make_uint2(br.lo, br.hi);
-        rsf[so] = (uint8_t)br.sf8;
+        if (rq) {                                     // (statistics-only callers pass no code buffers)
+          const BlockQ br = quantize_block(o, qc);
+          *reinterpret_cast<uint2*>(rq + qo) = make_uint2(br.lo, br.hi);
+          rsf[so] = (uint8_t)br.sf8;
+        }
       }
     }
     if (with_residual) {
@@ -1127,6 +1131,65 @@ export_site2_kernel(int A, int I, const int32_t* __restrict__ perm, const int32_
     *reinterpret_cast<uint2*>(r2q + (size_t)row * (I >> 1) + kb * 8) = v;
   }
   if (r2sf) r2sf[(size_t)row * k16 + kb] = r2sf_tiled[so];
+}
+
+
+// ---------------------------------------------------------------------------
+// Diagnostics of Eq. linear-mismatch: squared Frobenius norms of a - b, a and b for two bf16
+// tensors of equal size (two versions of a layer output), accumulated in float64 in a fixed order
+// (per-thread strided sums, warp tree, block tree, then the block partials in block order by
+// whichever CTA finishes last), so the three numbers are reproducible bit for bit.
+// `counter` must be zero on entry; out = {sum (a-b)^2, sum a^2, sum b^2}.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+mismatch_norms_kernel(const uint16_t* __restrict__ a, const uint16_t* __restrict__ b, int64_t n, double* __restrict__ partials,
+                      unsigned int* __restrict__ counter, double* __restrict__ out) {
+  pdl_sync();
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0;
+  const int64_t n8 = n >> 3;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
+    const uint4 va = __ldcs(reinterpret_cast<const uint4*>(a) + i), vb = __ldcs(reinterpret_cast<const uint4*>(b) + i);
+    float fa[8], fb[8];
+    unpack8(va, fa);
+    unpack8(vb, fb);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const double x = (double)fa[k], y = (double)fb[k], d = x - y;
+      s0 = fma(d, d, s0); s1 = fma(x, x, s1); s2 = fma(y, y, s2);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0)             // a tail that is not a multiple of 8 elements
+    for (int64_t i = n8 << 3; i < n; ++i) {
+      const double x = (double)bf16_bits_to_float(a[i]), y = (double)bf16_bits_to_float(b[i]), d = x - y;
+      s0 = fma(d, d, s0); s1 = fma(x, x, s1); s2 = fma(y, y, s2);
+    }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    s0 += __shfl_xor_sync(0xFFFFFFFFu, s0, o);
+    s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+    s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+  }
+  __shared__ double red[3][8];
+  __shared__ unsigned int last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { red[0][warp] = s0; red[1][warp] = s1; red[2][warp] = s2; }
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red[threadIdx.x][w];
+    partials[(size_t)blockIdx.x * 3 + threadIdx.x] = t;
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = atomicAdd(counter, 1u);
+  __syncthreads();
+  if (last == gridDim.x - 1 && threadIdx.x < 3) {
+    __threadfence();
+    double t = 0.0;
+    for (unsigned int g = 0; g < gridDim.x; ++g) t += __ldcg(partials + (size_t)g * 3 + threadIdx.x);
+    out[threadIdx.x] = t;
+  }
 }
 
 }  // namespace quads

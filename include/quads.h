@@ -77,11 +77,14 @@ size_t quads_sf_tiled_bytes(int64_t rows, int64_t K);
  *   gs_out out, float[1]: the per-tensor scale that was used (may be NULL)
  *   workspace  >= quads_quantize_workspace_bytes() bytes
  * rows == 0 is allowed (nothing is written except gs_out = 1 when gs_in is NULL).
- * With gs_in == NULL the kernel is one cooperative launch whose CTAs meet at a
- * counter once the tensor's amax is complete; that wait is bounded (about two
- * seconds).  If it ever gives up the call still ends, q and sf are unspecified
- * and gs_out[0] = NaN says so (pass gs_out to be able to tell); the same holds
- * for quads_fake_quant_activations.  With gs_in given there is no wait at all.
+ * With gs_in == NULL the call is two ordinary launches (per-CTA partial maxima,
+ * then the quantization, which finds the tensor in L2); with gs_in given it is
+ * one.  Neither contains a wait of one CTA for another.  (Setting the environment
+ * variable QUADS_QUANT_COOPERATIVE selects the single cooperative kernel that
+ * batches of large tensors use, whose CTAs meet at a counter once the amax is
+ * complete; that wait is bounded, about two seconds, and if it ever gives up
+ * the call still ends, q and sf are unspecified and gs_out[0] = NaN says so.)
+ * The same holds for quads_fake_quant_activations.
  * A tensor holds fewer than 2^31 scale blocks (rows * K / 16), else QUADS_ERR_SHAPE;
  * the same limit applies to every tensor of quads_fake_quant_weights.
  */
@@ -357,10 +360,10 @@ size_t quads_fp4_pipe_probe_operand_bytes(void);
 /*
  * Test hook (no counterpart in the paper): exercises the give-up path of a
  * bounded device-side wait without faulting or hanging anything.  It sets the
- * bound, in SM clock cycles, of the wait in which the CTAs of
- * quads_quantize_nvfp4 / quads_fake_quant_activations (and of
- * quads_fake_quant_weights when it takes the same kernel: one tensor, or
- * tensors above 32 MB) meet at a tensor's arrival counter in global memory, and
+ * bound, in SM clock cycles, of the wait in which the CTAs of the cooperative
+ * quantization kernel (quads_fake_quant_weights on tensors above 32 MB, or any
+ * quantizing call under QUADS_QUANT_COOPERATIVE / QUADS_NO_RING_QUANT) meet at a
+ * tensor's arrival counter in global memory, and
  * a surplus of arrivals to expect that nothing will ever deliver.  With a
  * surplus > 0 every such wait runs out after `clock_cycles`: the call still
  * completes, its outputs are unspecified and gs_out = NaN marks them.

@@ -139,7 +139,7 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
   L.header = take(kHdrWords * 4);
-  L.amax = take(16);
+  L.amax = take((size_t)kAmaxPartsMax * 4);    // the amax word; also the quantizer's scratch in the one-sided modes
   L.counters13 = take((size_t)((H + 31) / 32) * 4);
   L.counters2 = take((size_t)((I + 31) / 32 + 1) * 4);
   L.expert_total = take((size_t)Ee * 4);           // zeroed with the header: the routing kernel adds to it
@@ -307,9 +307,9 @@ size_t quads_sf_tiled_bytes(int64_t rows, int64_t K) {
   return (size_t)((rows + 127) / 128) * (size_t)((K + 63) / 64) * 512u;
 }
 
-size_t quads_quantize_workspace_bytes(void) { return 256; }
+size_t quads_quantize_workspace_bytes(void) { return (size_t)kAmaxPartsMax * 4; }
 size_t quads_fake_quant_workspace_bytes(int64_t n_tensors) {
-  return align_up((size_t)(n_tensors > 0 ? n_tensors : 1) * 8, 256);
+  return std::max(align_up((size_t)(n_tensors > 0 ? n_tensors : 1) * 8, 256), (size_t)kAmaxPartsMax * 4);
 }
 int32_t quads_last_launch_count(void) { return g_launch_count; }
 
@@ -342,8 +342,19 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   // scratch: one amax word and one arrival counter per tensor, zero on entry
   uint32_t* amax_bits = static_cast<uint32_t*>(workspace);
   uint32_t* counters = amax_bits + n_tensors;
-  if (!gs_in) QUADS_CUDA_OK(cudaMemsetAsync(amax_bits, 0, (size_t)n_tensors * 8, st));
   const uint16_t* xp = static_cast<const uint16_t*>(x);
+  // One tensor, scale to be derived: two ordinary launches instead of a cooperative one.  The first
+  // leaves one partial maximum per CTA in the workspace (no initialisation, no atomics) and asks L2 to
+  // keep the tensor; the second, launched as a programmatic dependent, reduces the partials and
+  // quantizes out of L2.  The kernel boundary is the only synchronisation.
+  const bool two_pass = !gs_in && n_tensors == 1 && rows > 0 && !getenv("QUADS_QUANT_COOPERATIVE");
+  if (!gs_in && !two_pass) QUADS_CUDA_OK(cudaMemsetAsync(amax_bits, 0, (size_t)n_tensors * 8, st));
+  int n_parts = 0;
+  if (two_pass) {
+    const int64_t chunks = rows * (K / 8);
+    n_parts = (int)std::max<int64_t>(1, std::min<int64_t>((chunks + 2047) / 2048, std::min(di.sm_count * 8, kAmaxPartsMax)));
+    QUADS_CUDA_OK(launch_kernel(amax_partial_kernel, dim3(n_parts), dim3(256), (size_t)0, st, xp, rows, K, ld, amax_bits));
+  }
   uint16_t* fqp = static_cast<uint16_t*>(fq);
   int nt = (int)n_tensors;
   int tiled = sf_layout == QUADS_SF_TILED;
@@ -403,11 +414,19 @@ static quads_status quantize_common(const void* x, int64_t n_tensors, int64_t ro
   if (grid < n_groups) grid = n_groups;
   long long wait_cycles = g_quant_wait_cycles.load();
   int extra_arrivals = g_quant_extra_arrivals.load();
-  void* args[] = {&xp, &rows, &K, &ld, &tensor_stride, &nt, &gs_in, &amax_bits, &counters, &q, &sf, &fqp,
-                  &gs_out, &tiled, &sf_stride, &n_groups, &wait_cycles, &extra_arrivals};
-  QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fused_quantize_kernel), dim3(grid), dim3(256),
-                                            args, 0, st));
-  note_launch();
+  const uint32_t* amax_parts = two_pass ? amax_bits : nullptr;
+  if (two_pass || gs_in) {
+    // no CTA waits for another one: an ordinary launch
+    QUADS_CUDA_OK(launch_kernel(fused_quantize_kernel, dim3(grid), dim3(256), (size_t)0, st, xp, rows, K, ld, tensor_stride, nt,
+                                gs_in, amax_bits, counters, q, sf, fqp, gs_out, tiled, sf_stride, n_groups, wait_cycles,
+                                extra_arrivals, amax_parts, n_parts));
+  } else {
+    void* args[] = {&xp, &rows, &K, &ld, &tensor_stride, &nt, &gs_in, &amax_bits, &counters, &q, &sf, &fqp,
+                    &gs_out, &tiled, &sf_stride, &n_groups, &wait_cycles, &extra_arrivals, &amax_parts, &n_parts};
+    QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fused_quantize_kernel), dim3(grid), dim3(256),
+                                              args, 0, st));
+    note_launch();
+  }
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
 }
@@ -715,7 +734,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     } else if (a->operand_mode == QUADS_W16A4) {
       // Q_A(x) then decode, in one pass of the quantizer (its scratch: the 256 bytes at the amax slot)
       const int launches = g_launch_count;
-      s = quantize_common(a->x, 1, T, H, H, 0, a->a13_gs, dec, a->xq, a->xsf, a->a13_gs_out, QUADS_SF_LINEAR, P(L.amax), 256, st);
+      s = quantize_common(a->x, 1, T, H, H, 0, a->a13_gs, dec, a->xq, a->xsf, a->a13_gs_out, QUADS_SF_LINEAR, P(L.amax), (size_t)kAmaxPartsMax * 4, st);
       g_launch_count += launches;
       if (s != QUADS_OK) return s;
       A_op = dec;

@@ -13,6 +13,8 @@ constexpr int kMaxExperts = 256;
 // header words written by the scan (device side sizes of the dispatch)
 enum { kHdrMTiles = 0, kHdrPaddedRows = 1, kHdrAssignments = 2, kHdrStatus = 3, kHdrArrivals = 4, kHdrWords = 8 };
 
+constexpr int kAmaxPartsMax = 2048;   // partial maxima left by the first pass of the single-tensor quantizer
+
 // ---- quantize.cu
 __global__ void amax_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, int64_t tensor_stride,
                             uint32_t* amax_bits);
@@ -20,7 +22,8 @@ __global__ void fused_quantize_kernel(const uint16_t* x, int64_t rows, int64_t K
                                       int n_tensors, const float* gs_in, uint32_t* amax_bits, uint32_t* counters,
                                       uint8_t* q, uint8_t* sf, uint16_t* fq, float* gs_out, int sf_tiled,
                                       int64_t sf_tensor_stride, int n_groups, long long wait_cycles,
-                                      int extra_arrivals);
+                                      int extra_arrivals, const uint32_t* amax_parts, int n_amax_parts);
+__global__ void amax_partial_kernel(const uint16_t* x, int64_t rows, int64_t K, int64_t ld, uint32_t* partials);
 // Fake-quant of a batch of tensors through shared-memory rings of bulk copies (one CTA per SM,
 // four groups of 7 consumer warps + 1 producer warp, one ring of 14 KB stages per group).
 constexpr int kRingThreads = 1024;

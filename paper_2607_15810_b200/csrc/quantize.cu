@@ -90,6 +90,46 @@ __device__ __forceinline__ uint32_t absmax8(const uint4& v) {
   return __vmaxu2(__vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu), __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu));
 }
 
+// First pass of the single-tensor quantizer: CTA b leaves the |x| maximum of its share in
+// partials[b] (every CTA stores, so the array needs no initialisation and there is no atomic);
+// the 32-byte loads ask L2 to keep the lines for the pass that follows.
+__global__ void __launch_bounds__(256) amax_partial_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K,
+                                                           int64_t ld, uint32_t* __restrict__ partials) {
+  pdl_sync();
+  const int64_t k16 = K >> 4, nblk = rows * k16;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  uint32_t m = 0;
+  int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (ld == K) {
+    for (; b + 3 * stride < nblk; b += 4 * stride) {
+      uint4 a0, a1, b0, b1, c0, c1, d0, d1;
+      ldg256_keep(x + b * 16, a0, a1);
+      ldg256_keep(x + (b + stride) * 16, b0, b1);
+      ldg256_keep(x + (b + 2 * stride) * 16, c0, c1);
+      ldg256_keep(x + (b + 3 * stride) * 16, d0, d1);
+      m = __vmaxu2(m, __vmaxu2(__vmaxu2(__vmaxu2(absmax8(a0), absmax8(a1)), __vmaxu2(absmax8(b0), absmax8(b1))),
+                               __vmaxu2(__vmaxu2(absmax8(c0), absmax8(c1)), __vmaxu2(absmax8(d0), absmax8(d1)))));
+    }
+  }
+  for (; b < nblk; b += stride) {
+    const int64_t r = b / k16, kb = b - r * k16;
+    uint4 a0, a1;
+    ldg256_keep(x + r * ld + kb * 16, a0, a1);
+    m = __vmaxu2(m, __vmaxu2(absmax8(a0), absmax8(a1)));
+  }
+  uint32_t sm = max(m & 0xFFFFu, m >> 16);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sm = max(sm, __shfl_xor_sync(0xFFFFFFFFu, sm, o));
+  __shared__ uint32_t wmax[8];
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = sm;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t t = 0;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t = max(t, wmax[i]);
+    partials[blockIdx.x] = t << 16;
+  }
+}
+
 // Where the quantizer's outputs of one tensor go (any pointer may be null).
 struct QuantSink {
   uint8_t* q;        // packed codes: block b owns bytes [8b, 8b+8)
@@ -144,7 +184,9 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
                       int n_tensors, const float* __restrict__ gs_in, uint32_t* __restrict__ amax_bits,
                       uint32_t* __restrict__ counters, uint8_t* __restrict__ q, uint8_t* __restrict__ sf,
                       uint16_t* __restrict__ fq, float* __restrict__ gs_out, int sf_tiled, int64_t sf_tensor_stride,
-                      int n_groups, long long wait_cycles, int extra_arrivals) {
+                      int n_groups, long long wait_cycles, int extra_arrivals, const uint32_t* __restrict__ amax_parts,
+                      int n_amax_parts) {
+  pdl_sync();
   const int group = blockIdx.x % n_groups;
   const int rank = blockIdx.x / n_groups;
   const int gsize = ((int)gridDim.x - group + n_groups - 1) / n_groups;
@@ -160,6 +202,22 @@ fused_quantize_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t K, i
     float gs;
     if (gs_in) {
       gs = gs_in[t];
+    } else if (amax_parts) {
+      // the tensor's amax was reduced to `n_amax_parts` partial maxima by the preceding kernel
+      uint32_t m = 0;
+      for (int i = threadIdx.x; i < n_amax_parts; i += blockDim.x) m = max(m, amax_parts[i]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+      if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        uint32_t tm = 0;
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) tm = max(tm, wmax[i]);
+        gs_sh = gs_from_amax_bits(tm);
+      }
+      __syncthreads();
+      gs = gs_sh;
+      __syncthreads();
     } else {
       // ---- phase 1: tensor amax, one 32-byte block per load
       uint32_t m = 0;

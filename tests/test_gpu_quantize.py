@@ -237,12 +237,13 @@ def test_aqat_layer_batch_at_full_size_against_the_oracle_on_sampled_tensors(B, 
         assert np.array_equal(F.bf16_bits(_f32(r["w_fq"][i])), F.bf16_bits(wf_o[0])), i
 
 
-def test_a_bounded_wait_that_runs_out_is_reported_and_harmless(B):
+def test_a_bounded_wait_that_runs_out_is_reported_and_harmless(B, monkeypatch):
     """Failure detection without a fault: the test hook makes the arrival wait of the quantize kernel
     expect one arrival more than there are CTAs and shortens its bound to about a millisecond.  The
     call must still end, mark its scale as NaN, and leave the library usable: the next ordinary call
     is bit-exact against the oracle."""
     x = _bf16((1, 16), 31, 2.0).cuda()
+    monkeypatch.setenv("QUADS_QUANT_COOPERATIVE", "1")        # the single-kernel path, whose CTAs wait for one another
     lib = B.lib
     lib.quads_debug_set_quantize_wait.restype = None
     lib.quads_debug_set_quantize_wait.argtypes = [B.C.c_int64, B.C.c_int32]
@@ -257,7 +258,11 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_harmless(B):
     finally:
         lib.quads_debug_set_quantize_wait(0, 0)
     big = _bf16((333, 2048), 3, 3.0)
-    q, sf, gs = B.quantize_nvfp4(big.cuda())
+    q, sf, gs = B.quantize_nvfp4(big.cuda())                   # still the cooperative kernel: intact after the give-up
+    c_o, s_o, g_o = Q.quantize(_f32(big))
+    assert np.float32(gs.item()) == g_o and np.array_equal(sf.cpu().numpy(), s_o)
+    monkeypatch.delenv("QUADS_QUANT_COOPERATIVE")
+    q, sf, gs = B.quantize_nvfp4(big.cuda())                   # and the default two-launch path
     c_o, s_o, g_o = Q.quantize(_f32(big))
     assert np.float32(gs.item()) == g_o and np.array_equal(sf.cpu().numpy(), s_o)
     assert np.array_equal(q.cpu().numpy(), F.pack_nibbles(c_o))

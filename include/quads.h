@@ -311,6 +311,48 @@ quads_status quads_moe_set_stage_trace(int32_t enable);
 int32_t quads_moe_get_stage_trace(const char** names /* host */, float* ms /* host */, int32_t cap);
 
 /*
+ * FP8 W8A8 comparison path: the "FP8 W8A8" rollout arm that the paper measures NVFP4 against
+ * (Section "Low-Precision Inference", paragraph FP8; Section "Rollout Throughput Comparison").  E4M3
+ * elements (maximum 448) with fine-grained power-of-two scales: one per (row, 128 channels) of an
+ * activation, one per 128 x 128 tile of a weight; scale = 2^e with e the smallest integer for which the
+ * tile's amax fits (amax <= 448 * 2^e), stored as the byte e + 127; element = E4M3_rne_sat(x * 2^-e).
+ * The same MoE layer as quads_moe_w4a4_rac (top-k routing, dispatch order, SwiGLU, h rounded to bf16
+ * and requantized per (row, 128 features), weighted combine) on block-scaled FP8 tensor-core GEMMs;
+ * there is no residual compensation in this format.
+ *
+ * quads_fp8_quantize_weights:  w bf16 [n, N, K] (N % 128 == 0, K % 128 == 0, 16-byte aligned) ->
+ *   q u8 [n, N, K], exps u8 [n, N/128, K/128], atoms u8 [n, N/128, K/128, 512] (each tile's scale byte
+ *   repeated 512 times: what the GEMM copies into tensor memory; 16-byte aligned).
+ * quads_moe_fp8_w8a8: H % 128 == 0, I % 128 == 0, limits on E / topk as for quads_moe_w4a4_rac; the
+ *   optional exports (dispatch order, A = T * topk rows) serve verification.  Enqueued on one stream;
+ *   device-side waits are bounded and report through quads_moe_async_status(workspace).
+ */
+quads_status quads_fp8_quantize_weights(const void* w, int64_t n_tensors, int64_t N, int64_t K, uint8_t* q,
+                                        uint8_t* exps, uint8_t* atoms, void* cuda_stream);
+typedef struct {
+  int32_t T, H, I, E, topk;
+  const void* x;                 /* bf16 [T, H] */
+  const float* router_logits;    /* float [T, E] */
+  const uint8_t* w13_q;          /* u8 [E, 2I, H], gate rows first */
+  const uint8_t* w13_atoms;      /* u8 [E, 2I/128, H/128, 512] */
+  const uint8_t* w2_q;           /* u8 [E, H, I] */
+  const uint8_t* w2_atoms;       /* u8 [E, H/128, I/128, 512] */
+  int32_t renormalize;
+  void* out;                     /* bf16 [T, H] */
+  int32_t* topk_ids;             /* optional exports: [T, topk] */
+  int32_t* perm;                 /* [A] */
+  uint8_t* xq;                   /* [T, H] E4M3 codes of x, token order */
+  uint8_t* xexp;                 /* [T, H/128] */
+  void* h_bf16;                  /* bf16 [A, I]; with it hq [A, I] and hexp [A, I/128] must be given too */
+  uint8_t* hq;
+  uint8_t* hexp;
+  void* workspace;
+  size_t workspace_bytes;        /* >= quads_moe_fp8_workspace_bytes(T, H, I, E, topk), 256-byte aligned */
+} quads_moe_fp8_args;
+quads_status quads_moe_fp8_w8a8(const quads_moe_fp8_args* args /* host */, void* cuda_stream);
+size_t quads_moe_fp8_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk);
+
+/*
  * Diagnostics of the paper's mismatch analysis, computed on the device.
  *
  * quads_rac_channel_scores: s_j^2 = sum over the token batch of (Q_A(X) - X)[:, j]^2, the squared

@@ -380,3 +380,71 @@ def mismatch_norms(a, b, workspace=None):
     ws = workspace if workspace is not None else _ws(lib.quads_mismatch_norms_workspace_bytes(), a.device)
     check(lib.quads_mismatch_norms(_ptr(a), _ptr(b), a.numel(), _ptr(out), _ptr(ws), ws.numel(), _stream()))
     return out
+
+
+class MoEFp8Args(C.Structure):
+    _fields_ = [
+        ("T", _i32), ("H", _i32), ("I", _i32), ("E", _i32), ("topk", _i32),
+        ("x", _p), ("router_logits", _p),
+        ("w13_q", _p), ("w13_atoms", _p), ("w2_q", _p), ("w2_atoms", _p),
+        ("renormalize", _i32),
+        ("out", _p),
+        ("topk_ids", _p), ("perm", _p), ("xq", _p), ("xexp", _p), ("h_bf16", _p), ("hq", _p), ("hexp", _p),
+        ("workspace", _p), ("workspace_bytes", _sz),
+    ]
+
+
+lib.quads_fp8_quantize_weights.restype = _i32
+lib.quads_fp8_quantize_weights.argtypes = [_p, _i64, _i64, _i64, _p, _p, _p, _p]
+lib.quads_moe_fp8_w8a8.restype = _i32
+lib.quads_moe_fp8_w8a8.argtypes = [C.POINTER(MoEFp8Args), _p]
+lib.quads_moe_fp8_workspace_bytes.restype = _sz
+lib.quads_moe_fp8_workspace_bytes.argtypes = [_i32] * 5
+
+
+def fp8_quantize_weights(w):
+    """w: bf16 CUDA [n, N, K] -> dict(q u8 [n, N, K], exps u8 [n, N/128, K/128], atoms u8 [n, N/128, K/128, 512])."""
+    assert w.dtype == torch.bfloat16 and w.is_cuda and w.dim() == 3 and w.is_contiguous()
+    n, N, K = w.shape
+    dev = w.device
+    q = torch.empty(n, N, K, dtype=torch.uint8, device=dev)
+    exps = torch.empty(n, N // 128, K // 128, dtype=torch.uint8, device=dev)
+    atoms = torch.empty(n, N // 128, K // 128, 512, dtype=torch.uint8, device=dev)
+    check(lib.quads_fp8_quantize_weights(_ptr(w), n, N, K, _ptr(q), _ptr(exps), _ptr(atoms), _stream()))
+    return dict(q=q, exps=exps, atoms=atoms)
+
+
+def moe_fp8_workspace_bytes(T, H, I, E, topk):
+    return lib.quads_moe_fp8_workspace_bytes(T, H, I, E, topk)
+
+
+def moe_fp8_w8a8(x, logits, w13, w2, topk, renormalize=True, export=False, workspace=None, out=None):
+    """FP8 W8A8 MoE layer (comparison path).  w13 / w2: dicts from fp8_quantize_weights."""
+    T, H = x.shape
+    E = logits.shape[1]
+    I = w2["q"].shape[2]
+    dev = x.device
+    A = T * topk
+    a = MoEFp8Args()
+    a.T, a.H, a.I, a.E, a.topk = T, H, I, E, topk
+    a.x, a.router_logits = _ptr(x), _ptr(logits)
+    a.w13_q, a.w13_atoms, a.w2_q, a.w2_atoms = _ptr(w13["q"]), _ptr(w13["atoms"]), _ptr(w2["q"]), _ptr(w2["atoms"])
+    a.renormalize = 1 if renormalize else 0
+    res = {"out": out if out is not None else torch.empty(T, H, dtype=torch.bfloat16, device=dev)}
+    a.out = _ptr(res["out"])
+    if export:
+        u8 = torch.uint8
+        res["ids"] = torch.empty(T, topk, dtype=torch.int32, device=dev)
+        res["perm"] = torch.empty(A, dtype=torch.int32, device=dev)
+        res["xq"] = torch.empty(T, H, dtype=u8, device=dev)
+        res["xexp"] = torch.empty(T, H // 128, dtype=u8, device=dev)
+        res["h"] = torch.empty(A, I, dtype=torch.bfloat16, device=dev)
+        res["hq"] = torch.empty(A, I, dtype=u8, device=dev)
+        res["hexp"] = torch.empty(A, I // 128, dtype=u8, device=dev)
+        a.topk_ids, a.perm, a.xq, a.xexp = map(_ptr, (res["ids"], res["perm"], res["xq"], res["xexp"]))
+        a.h_bf16, a.hq, a.hexp = map(_ptr, (res["h"], res["hq"], res["hexp"]))
+    ws = workspace if workspace is not None else _ws(moe_fp8_workspace_bytes(T, H, I, E, topk), dev)
+    a.workspace, a.workspace_bytes = _ptr(ws), ws.numel()
+    check(lib.quads_moe_fp8_w8a8(C.byref(a), _stream()))
+    res["workspace"] = ws
+    return res

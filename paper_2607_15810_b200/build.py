@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libquads.so")
-SOURCES = ["api.cu", "quantize.cu", "routing.cu", "gemm.cu", "gemm_swapped.cu", "gemm_bf16.cu", "probe.cu"]
+SOURCES = ["api.cu", "quantize.cu", "routing.cu", "gemm.cu", "gemm_swapped.cu", "gemm_bf16.cu", "fp8.cu", "probe.cu"]
 HEADERS = ["common.cuh", "kernels.cuh", "tcgen05.cuh", os.path.join("..", "..", "include", "quads.h")]
 
 

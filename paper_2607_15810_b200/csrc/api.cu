@@ -978,4 +978,167 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   return QUADS_OK;
 }
 
+
+// ---------------------------------------------------------------------------
+// FP8 W8A8 comparison path
+// ---------------------------------------------------------------------------
+namespace {
+struct Fp8Layout {
+  size_t header, expert_total, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
+  size_t perm, pos_pad, row_token, row_weight, xq_tok, xe_tok, xq_pad, xsf, hq_pad, hsf, y_pad, total;
+  int n_chunks, m_tiles_max;
+};
+Fp8Layout fp8_layout(int T, int H, int I, int E, int topk) {
+  Fp8Layout L{};
+  const int64_t A = (int64_t)T * topk;
+  L.n_chunks = (T + kRouteTokensPerCta - 1) / kRouteTokensPerCta;
+  L.m_tiles_max = (int)(A / 128) + E;
+  const size_t pad_rows = (size_t)L.m_tiles_max * 128;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+  L.header = take(kHdrWords * 4);
+  L.expert_total = take((size_t)E * 4);
+  L.ids = take((size_t)A * 4);
+  L.wts = take((size_t)A * 4);
+  L.chunk_counts = take((size_t)L.n_chunks * E * 4);
+  L.chunk_base = take((size_t)L.n_chunks * E * 4);
+  L.offsets = take((size_t)(E + 1) * 4);
+  L.tile_prefix = take((size_t)(E + 1) * 4);
+  L.tile_expert = take((size_t)L.m_tiles_max * 4);
+  L.tile_rows = take((size_t)L.m_tiles_max * 4);
+  L.perm = take((size_t)A * 4);
+  L.pos_pad = take((size_t)A * 4);
+  L.row_token = take(pad_rows * 4);
+  L.row_weight = take(pad_rows * 4);
+  L.xq_tok = take((size_t)T * H);
+  L.xe_tok = take((size_t)T * (H / 128));
+  L.xq_pad = take(pad_rows * (size_t)H);
+  L.xsf = take((size_t)L.m_tiles_max * (H / 128) * 512);
+  L.hq_pad = take(pad_rows * (size_t)I);
+  L.hsf = take((size_t)L.m_tiles_max * (I / 128) * 512);
+  L.y_pad = take(pad_rows * (size_t)H * 2);
+  L.total = o;
+  return L;
+}
+}  // namespace
+
+quads_status quads_fp8_quantize_weights(const void* w, int64_t n_tensors, int64_t N, int64_t K, uint8_t* q,
+                                        uint8_t* exps, uint8_t* atoms, void* cuda_stream) {
+  g_launch_count = 0;
+  if (n_tensors < 0 || N <= 0 || K <= 0 || (N % 128) != 0 || (K % 128) != 0) return QUADS_ERR_SHAPE;
+  if (n_tensors * (N / 128) * (K / 128) > (int64_t)0x7FFFFFFF) return QUADS_ERR_SHAPE;
+  if (n_tensors == 0) return QUADS_OK;
+  if (!w || !q || !exps || !atoms) return QUADS_ERR_NULL;
+  if (!aligned(w, 16) || !aligned(q, 16) || !aligned(atoms, 16)) return QUADS_ERR_SHAPE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  const unsigned grid = (unsigned)(n_tensors * (N / 128) * (K / 128));
+  QUADS_CUDA_OK(launch_kernel(fp8_quantize_weight_kernel, dim3(grid), dim3(256), (size_t)0, static_cast<cudaStream_t>(cuda_stream),
+                              static_cast<const uint16_t*>(w), (int)N, (int)K, q, exps, atoms));
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
+size_t quads_moe_fp8_workspace_bytes(int32_t T, int32_t H, int32_t I, int32_t E, int32_t topk) {
+  if (T < 0 || H <= 0 || I <= 0 || E < 1 || topk < 1) return 0;
+  return fp8_layout(T, H, I, E, topk).total;
+}
+
+
+quads_status quads_moe_fp8_w8a8(const quads_moe_fp8_args* a, void* cuda_stream) {
+  g_launch_count = 0;
+  if (!a) return QUADS_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int T = a->T, H = a->H, I = a->I, E = a->E, topk = a->topk;
+  if (T < 0 || H <= 0 || (H % 128) != 0 || I <= 0 || (I % 128) != 0 || H > 16384 || I > 16384) return QUADS_ERR_SHAPE;
+  if (E < 1 || E > kMaxExperts || topk < 1 || topk > kMaxTopk || topk > E) return QUADS_ERR_SHAPE;
+  if ((int64_t)T * topk > 0x3FFFFFFF) return QUADS_ERR_SHAPE;
+  if (T == 0) return QUADS_OK;
+  if (!a->x || !a->router_logits || !a->w13_q || !a->w13_atoms || !a->w2_q || !a->w2_atoms || !a->out) return QUADS_ERR_NULL;
+  if (a->h_bf16 && (!a->hq || !a->hexp)) return QUADS_ERR_NULL;
+  if (!aligned(a->x, 16) || !aligned(a->w13_q, 16) || !aligned(a->w13_atoms, 16) || !aligned(a->w2_q, 16) ||
+      !aligned(a->w2_atoms, 16) || !aligned(a->out, 16) || !aligned(a->h_bf16, 16) || !aligned(a->hq, 16))
+    return QUADS_ERR_SHAPE;
+  const Fp8Layout L = fp8_layout(T, H, I, E, topk);
+  if (!a->workspace || !aligned(a->workspace, 256) || a->workspace_bytes < L.total) return QUADS_ERR_WORKSPACE;
+  DeviceInfo di;
+  quads_status s = device_info(&di);
+  if (s != QUADS_OK) return s;
+  uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+  auto P = [&](size_t off) { return ws + off; };
+  int32_t* header = reinterpret_cast<int32_t*>(P(L.header));
+  int32_t* ids = reinterpret_cast<int32_t*>(P(L.ids));
+  float* wts = reinterpret_cast<float*>(P(L.wts));
+  int32_t* chunk_counts = reinterpret_cast<int32_t*>(P(L.chunk_counts));
+  int32_t* chunk_base = reinterpret_cast<int32_t*>(P(L.chunk_base));
+  int32_t* expert_total = reinterpret_cast<int32_t*>(P(L.expert_total));
+  int32_t* offsets = reinterpret_cast<int32_t*>(P(L.offsets));
+  int32_t* tile_prefix = reinterpret_cast<int32_t*>(P(L.tile_prefix));
+  int32_t* tile_expert = reinterpret_cast<int32_t*>(P(L.tile_expert));
+  int32_t* tile_rows = reinterpret_cast<int32_t*>(P(L.tile_rows));
+  int32_t* perm = reinterpret_cast<int32_t*>(P(L.perm));
+  int32_t* pos_pad = reinterpret_cast<int32_t*>(P(L.pos_pad));
+  int32_t* row_token = reinterpret_cast<int32_t*>(P(L.row_token));
+  float* row_weight = reinterpret_cast<float*>(P(L.row_weight));
+  const size_t pad_rows = (size_t)L.m_tiles_max * 128;
+  QUADS_CUDA_OK(cudaMemsetAsync(ws, 0, L.ids, st));            // header, status word, per-expert totals
+  // ---- routing and dispatch order (the NVFP4 path's kernels)
+  {
+    auto route = E <= 32 ? route_kernel_t<1> : (E <= 64 ? route_kernel_t<2> : (E <= 128 ? route_kernel_t<4> : route_kernel_t<8>));
+    QUADS_CUDA_OK(launch_kernel(route, dim3(L.n_chunks), dim3(256), (size_t)0, st, a->router_logits, T, E, topk, a->renormalize,
+                                ids, wts, chunk_counts, expert_total, a->topk_ids, (float*)nullptr));
+  }
+  QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(E), dim3(256), (size_t)0, st, E, L.n_chunks, 1, chunk_counts, expert_total,
+                              chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, (int32_t*)nullptr));
+  QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3(L.n_chunks), dim3(128), (size_t)0, st, T, E, topk, L.n_chunks, ids, wts,
+                              chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
+  // ---- activation quantization (token order) and dispatch
+  uint8_t* xq_tok = a->xq ? a->xq : P(L.xq_tok);
+  uint8_t* xe_tok = a->xexp ? a->xexp : P(L.xe_tok);
+  {
+    const int64_t tiles = (int64_t)T * (H / 128);
+    const unsigned grid = (unsigned)std::min<int64_t>((tiles + 7) / 8, (int64_t)di.sm_count * 16);
+    QUADS_CUDA_OK(launch_kernel(fp8_quantize_act_kernel, dim3(grid), dim3(256), (size_t)0, st, static_cast<const uint16_t*>(a->x),
+                                (int64_t)T, H, xq_tok, xe_tok));
+  }
+  QUADS_CUDA_OK(launch_kernel(fp8_dispatch_kernel, dim3(L.m_tiles_max), dim3(256), (size_t)0, st, H, header, tile_rows, row_token,
+                              xq_tok, xe_tok, P(L.xq_pad), P(L.xsf)));
+  // ---- first projection: W13, SwiGLU, requantize
+  CUtensorMap ma, mb;
+  if ((s = make_codes_map(&ma, P(L.xq_pad), pad_rows, (uint64_t)H)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&mb, a->w13_q, (uint64_t)E * 2 * I, (uint64_t)H)) != QUADS_OK) return s;
+  Fp8GemmParams g{};
+  g.K = H; g.n_tiles_n = I / 128; g.n_out = I; g.b_rows_per_expert = 2 * I; g.half1_row_offset = I;
+  g.header = header; g.tile_expert = tile_expert; g.tile_rows = tile_rows;
+  g.a_sf = P(L.xsf); g.b_sf = a->w13_atoms; g.b_sf_expert_stride = (size_t)(2 * I / 128) * (H / 128) * 512;
+  g.hq_pad = P(L.hq_pad); g.hsf_atoms = P(L.hsf);
+  g.h_export = static_cast<uint16_t*>(a->h_bf16); g.hq_export = a->hq; g.hexp_export = a->hexp;
+  g.tile_prefix = tile_prefix; g.offsets = offsets; g.status = header + kHdrStatus;
+  const bool timing = g_timers.enabled && g_timers.created;
+  if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[0], st));
+  if ((s = launch_gemm_fp8(kEpiSwiGLU, g, ma, mb, di.sm_count, st)) != QUADS_OK) return s;
+  if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[1], st));
+  // ---- second projection and weighted combine
+  CUtensorMap m2a, m2b;
+  if ((s = make_codes_map(&m2a, P(L.hq_pad), pad_rows, (uint64_t)I)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m2b, a->w2_q, (uint64_t)E * H, (uint64_t)I)) != QUADS_OK) return s;
+  Fp8GemmParams g2 = g;
+  g2.K = I; g2.n_tiles_n = (H + 255) / 256; g2.n_out = H; g2.b_rows_per_expert = H; g2.half1_row_offset = 128;
+  g2.a_sf = P(L.hsf); g2.b_sf = a->w2_atoms; g2.b_sf_expert_stride = (size_t)(H / 128) * (I / 128) * 512;
+  g2.y_pad = reinterpret_cast<uint16_t*>(P(L.y_pad));
+  g2.h_export = nullptr;
+  if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[2], st));
+  if ((s = launch_gemm_fp8(kEpiCombine, g2, m2a, m2b, di.sm_count, st)) != QUADS_OK) return s;
+  if (timing) {
+    QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[3], st));
+    g_timers.valid = true;
+  }
+  const int64_t n8 = (int64_t)T * (H / 8);
+  QUADS_CUDA_OK(launch_kernel(combine_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), (size_t)0, st, g2.y_pad, pos_pad, wts,
+                              T, H, topk, static_cast<uint16_t*>(a->out)));
+  QUADS_CUDA_OK(cudaGetLastError());
+  return QUADS_OK;
+}
+
 }  // extern "C"

@@ -118,45 +118,6 @@ __device__ __forceinline__ float warp_colsum16(const float* v, int lane) {
   return d;
 }
 
-__device__ __forceinline__ void stg256(void* addr, const uint32_t* v) {
-  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]),
-               "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
-}
-
-// Store a warp's 32 rows x 64 accumulator columns (thread = row) as bf16, scaled, to rows of
-// `n_out` elements starting at `dst`, rows >= rows_valid skipped.  The 32-byte chunks are first
-// transposed inside every group of 4 lanes (two butterfly exchanges), so that each store
-// instruction of the warp writes eight complete 128-byte lines instead of a 32-byte piece of 32
-// different lines.  All 32 lanes must call it.
-__device__ __forceinline__ void store_y_rows(const float* acc, float scale, uint16_t* dst, int n_out, int rows_valid,
-                                             int lane) {
-  uint32_t w[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) w[i] = f32x2_to_bf16x2(acc[2 * i] * scale, acc[2 * i + 1] * scale);
-  // chunk c = w[8c .. 8c+7]; after the exchanges chunk slot c of lane (g, j) holds chunk j of lane (g, c)
-#pragma unroll
-  for (int s = 1; s < 4; s <<= 1) {
-    const bool up = (lane & s) != 0;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      if (c & s) continue;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const uint32_t lo = w[8 * c + k], hi = w[8 * (c | s) + k];
-        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, up ? lo : hi, s);
-        w[8 * c + k] = up ? got : lo;
-        w[8 * (c | s) + k] = up ? hi : got;
-      }
-    }
-  }
-  const int g = lane >> 2, j = lane & 3;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = 4 * g + i;
-    if (r < rows_valid) stg256(dst + (size_t)r * n_out + 16 * j, w + 8 * i);
-  }
-}
-
 template <int EPI, int CG>
 __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap* tm_a, const CUtensorMap* tm_r,
                                           const CUtensorMap* tm_b, const CUtensorMap* tm_sfa,

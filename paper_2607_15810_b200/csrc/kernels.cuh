@@ -141,6 +141,36 @@ quads_status launch_gemm_swapped(int epi, const GemmParams& p, const GemmMaps& m
 quads_status launch_gemm_bf16(const CUtensorMap& tm_a, const CUtensorMap& tm_b, int T, int N, int K, uint16_t* out,
                               int32_t* status, int n_sms, cudaStream_t stream);
 
+// ---- fp8.cu: the FP8 W8A8 comparison path
+struct Fp8GemmParams {
+  int K;                 // contraction length in elements (multiple of 128)
+  int n_tiles_n;         // tiles along the output features
+  int n_out;             // output features (I for SwiGLU, else H)
+  int b_rows_per_expert;
+  int half1_row_offset;
+  const int32_t* header;
+  const int32_t* tile_expert;
+  const int32_t* tile_rows;
+  const uint8_t* a_sf;   // activation scale atoms, [m_tiles, K/128, 512]
+  const uint8_t* b_sf;   // weight scale atoms, [E, rows/128, K/128, 512]
+  size_t b_sf_expert_stride;
+  uint16_t* y_pad;       // kEpiCombine: bf16 [padded rows, n_out]
+  uint8_t* hq_pad;       // kEpiSwiGLU: E4M3 codes of h, [padded rows, n_out]
+  uint8_t* hsf_atoms;    // kEpiSwiGLU: scale atoms of h, [m_tiles, n_out/128, 512]
+  uint16_t* h_export;    // optional bf16 [A, n_out], dispatch order (then hq_export / hexp_export too)
+  uint8_t* hq_export;
+  uint8_t* hexp_export;
+  const int32_t* tile_prefix;
+  const int32_t* offsets;
+  int32_t* status;
+};
+__global__ void fp8_quantize_act_kernel(const uint16_t* x, int64_t rows, int K, uint8_t* codes, uint8_t* exps);
+__global__ void fp8_quantize_weight_kernel(const uint16_t* w, int N, int K, uint8_t* codes, uint8_t* exps, uint8_t* atoms);
+__global__ void fp8_dispatch_kernel(int H, const int32_t* header, const int32_t* tile_rows, const int32_t* row_token,
+                                    const uint8_t* xq, const uint8_t* xe, uint8_t* xq_pad, uint8_t* xsf_atoms);
+quads_status launch_gemm_fp8(int epi, const Fp8GemmParams& p, const CUtensorMap& tm_a, const CUtensorMap& tm_b, int n_sms,
+                             cudaStream_t stream);
+
 quads_status launch_gemm(int epi, int cta_group, const GemmParams& p, const GemmMaps& m, int n_sms,
                          cudaStream_t stream);
 

@@ -180,6 +180,15 @@ class ClockSampler:
                 pass
             time.sleep(self.period)
 
+    def pcie(self):
+        """Current PCIe link generation and width (the bound of the end-to-end number), read only."""
+        try:
+            nv = self.nv
+            return {"gen": int(nv.nvmlDeviceGetCurrPcieLinkGeneration(self.h)), "width": int(nv.nvmlDeviceGetCurrPcieLinkWidth(self.h)),
+                    "max_gen": int(nv.nvmlDeviceGetMaxPcieLinkGeneration(self.h)), "max_width": int(nv.nvmlDeviceGetMaxPcieLinkWidth(self.h))}
+        except Exception:
+            return None
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
         if self._thread is None:
@@ -421,6 +430,7 @@ def run_ours(args):
     barrier()
     e2e_pipe_ms = max_over_ranks(pipelined(args.steps))
     barrier()
+    pcie = sampler.pcie() if sampler else None
     clocks = sampler.stop() if sampler else None
 
     # per-kernel time of the two grouped GEMMs (events recorded by the library on the launch stream)
@@ -475,7 +485,8 @@ def run_ours(args):
                     "h2d_bytes_per_step": x_h.numel() * 2 + lg_h.numel() * 4, "d2h_bytes_per_step": out_h.numel() * 2,
                     "how": "every step copies its inputs from pinned host memory and its result back; copies run on "
                            "their own streams with two device buffers each way, so they overlap neighbouring steps",
-                    "serial_value": D.whole_job_rate(world, T, e2e_ms), "serial_ms_per_step": e2e_ms},
+                    "serial_value": D.whole_job_rate(world, T, e2e_ms), "serial_ms_per_step": e2e_ms,
+                    "pcie_link": pcie},
             "gpu_launches": launches_per_step * args.steps,
             "tflops": {"model": f_model / (ms * 1e-3) / 1e12, "algorithmic": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12,
                        "frac_of_fp4_peak": (f_alg1 + f_alg2) / (ms * 1e-3) / 1e12 / fp4_peak},

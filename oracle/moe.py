@@ -114,7 +114,8 @@ def _absdot(site, w_abs):
 
 
 def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
-                a13_gs=None, renormalize=True, forced_sel13=None, forced_sel2=None, h_override=None):
+                a13_gs=None, renormalize=True, forced_sel13=None, forced_sel2=None, h_override=None,
+                expert_range=None):
     """MoE layer forward.
       x       float32 (bf16-valued) [T, H]
       logits  float32 [T, E]
@@ -127,6 +128,12 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
               first halves that differ by one bf16 ulp give different (both
               valid) codes; the staged comparison checks the second half of
               an implementation on that implementation's own h.
+      expert_range  (lo, hi): expert-sharded execution.  Only the contributions of experts lo..hi-1 are
+              computed (w13 / w2 still hold all experts here): routing and site 13 are those of the whole
+              layer, h / site 2 cover the shard's dispatched rows offsets[lo]..offsets[hi] only (its own
+              "current token batch" for the site-2 scores), out64 is the shard's partial sum.  The
+              partial sums of disjoint shards that cover all experts add up to the layer output when
+              site 2 is not compensated; with site-2 RAC every shard selects on its own rows.
     Returns a dict of every intermediate the CUDA path can export."""
     x = np.asarray(x, dtype=F32)
     T, H = x.shape
@@ -145,10 +152,12 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
           + np.abs(Q.dequantize_real(site13["r_codes"], site13["r_sf"], site13["r_gs"])))
 
     tok_of = perm // topk                                  # token of each dispatched row
-    h64 = np.empty((A, I), dtype=np.float64)
-    g64 = np.empty((A, 2 * I), dtype=np.float64)
-    g_absdot = np.empty((A, 2 * I), dtype=np.float64)
-    for e in range(E):
+    e_lo, e_hi = (0, E) if expert_range is None else expert_range
+    row_lo, row_hi = int(offsets[e_lo]), int(offsets[e_hi])
+    h64 = np.zeros((A, I), dtype=np.float64)
+    g64 = np.zeros((A, 2 * I), dtype=np.float64)
+    g_absdot = np.zeros((A, 2 * I), dtype=np.float64)
+    for e in range(e_lo, e_hi):
         lo, hi = offsets[e], offsets[e + 1]
         if lo == hi:
             continue
@@ -158,10 +167,12 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
         g64[lo:hi] = g
         g_absdot[lo:hi] = xa[rows] @ np.abs(w).T
         h64[lo:hi] = silu(g[:, :I]) * g[:, I:]
-    h = F.bf16_round(h64)                                  # [A, I] in dispatch order
+    h = F.bf16_round(h64)[row_lo:row_hi]                   # the shard's rows of [A, I], dispatch order
+    g64, g_absdot, h64 = g64[row_lo:row_hi], g_absdot[row_lo:row_hi], h64[row_lo:row_hi]
     h_own = h
     if h_override is not None:
         h = np.asarray(h_override, dtype=F32)
+        assert h.shape == h_own.shape
 
     # ---- site 2: all A dispatched rows together are the batch
     site2 = R.rac(h, n_sel2, a2_gs, None)
@@ -174,13 +185,13 @@ def moe_forward(x, logits, w13, w2, topk, n_sel13, n_sel2, a2_gs,
     out64 = np.zeros((T, H), dtype=np.float64)
     out_absdot = np.zeros((T, H), dtype=np.float64)
     w_flat = wts.reshape(-1).astype(np.float64)
-    for e in range(E):
+    for e in range(e_lo, e_hi):
         lo, hi = offsets[e], offsets[e + 1]
         if lo == hi:
             continue
         w = Q.dequantize_real(w2["codes"][e], w2["sf"][e], w2["gs"][e])      # [H, I]
-        y = ht[lo:hi] @ w.T
-        ya = ha[lo:hi] @ np.abs(w).T
+        y = ht[lo - row_lo:hi - row_lo] @ w.T
+        ya = ha[lo - row_lo:hi - row_lo] @ np.abs(w).T
         gw = w_flat[perm[lo:hi]][:, None]
         rows = tok_of[lo:hi]                 # distinct: a token picks an expert at most once
         assert np.unique(rows).size == rows.size

@@ -436,3 +436,38 @@ def test_one_sided_modes_against_loops_and_their_special_cases():
     assert np.array_equal(M.dense_w4a16(xe, cw, sw, gw)["y64"], plain)
     assert np.array_equal(M.dense_w16a4(xe, we)["y64"], plain)
     assert np.array_equal(M.dense_w4a4_rac(xe, cw, sw, gw, 0)["y64"], plain)
+
+
+def test_expert_sharded_oracle_adds_up_to_the_layer():
+    """Expert-sharded execution: routing and site 13 are the layer's; a shard's rows are its experts'
+    segment of the dispatch order; without site-2 compensation the shards' partial sums add up to the
+    layer output, and with it every shard runs RAC on its own rows."""
+    x, logits, w13, w2, a2 = _two_expert_case()                 # three experts, two slots
+    full0 = M.moe_forward(x, logits, w13, w2, 2, 16, 0, a2)
+    parts = [M.moe_forward(x, logits, w13, w2, 2, 16, 0, a2, expert_range=r) for r in ((0, 1), (1, 3))]
+    assert np.allclose(parts[0]["out64"] + parts[1]["out64"], full0["out64"], rtol=1e-12, atol=1e-15)
+    off = full0["offsets"]
+    for p, (lo, hi) in zip(parts, ((0, 1), (1, 3))):
+        assert np.array_equal(p["site13"]["r_codes"], full0["site13"]["r_codes"])
+        assert np.array_equal(p["h"], full0["h"][off[lo]:off[hi]])
+        assert np.array_equal(p["g64"], full0["g64"][off[lo]:off[hi]])
+    # with site-2 RAC: the shard's site 2 is RAC on its own rows, and its partial output follows from it
+    sh = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, expert_range=(1, 3))
+    want = R.rac(full0["h"][off[1]:off[3]], 8, a2)
+    for k in ("codes", "sf", "r_codes", "r_sf", "sel"):
+        assert np.array_equal(sh["site2"][k], want[k]), k
+    ht = R.reconstruct_real(want)
+    inv = np.empty(18, int)
+    inv[full0["perm"]] = np.arange(18)
+    ref = np.zeros((9, 32))
+    for t in range(9):
+        for s in range(2):
+            e = int(full0["ids"][t, s])
+            if e in (1, 2):
+                w2e = _scalar_dequant(w2["codes"][e], w2["sf"][e], w2["gs"][e])
+                ref[t] += float(full0["weights"][t, s]) * _triple_loop([ht[inv[t * 2 + s] - off[1]].tolist()], w2e.tolist())[0]
+    assert np.allclose(sh["out64"], ref, rtol=1e-11, atol=1e-14)
+    # a whole-range shard is the layer itself
+    whole = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2, expert_range=(0, 3))
+    full = M.moe_forward(x, logits, w13, w2, 2, 16, 8, a2)
+    assert np.array_equal(whole["out64"], full["out64"]) and np.array_equal(whole["site2"]["r_codes"], full["site2"]["r_codes"])

@@ -276,8 +276,18 @@ typedef struct {
   /* Dense mode only: which operands are NVFP4 (the one-sided rollout modes of Table
      "qdq-alignment" and Section "Train-inference mismatch ...").  Modes 1 and 2 take no RAC
      (rac_nsel_13 must be 0): they exist to isolate one side's quantization error. */
-  int32_t operand_mode;         /* QUADS_W4A4 (0, default), QUADS_W4A16 or QUADS_W16A4 */
-  const void* w13_bf16;         /* QUADS_W16A4: the unquantized weight, bf16 [N, H], 16-byte aligned */
+  int32_t operand_mode;         /* QUADS_W4A4 (0, default), QUADS_W4A16, QUADS_W16A4 or QUADS_W16A16 */
+  const void* w13_bf16;         /* QUADS_W16A4 / QUADS_W16A16: the unquantized weight, bf16 [N, H], 16-byte aligned */
+  /* Expert-sharded execution (MoE mode; the paper's engines run the experts expert-parallel, Section
+     "Experimental setup"): this call holds the weights of experts [expert_lo, expert_lo + expert_count)
+     only -- w13_* / w2_* are arrays over those experts -- while x, router_logits and the routing are
+     those of the whole layer (E experts).  It computes the contributions of its experts to every token:
+     quantization, channel statistics and both selections run over the whole token batch at site 13
+     (identical on every shard) and over the shard's own dispatched rows at site 2.  The partial sums are
+     written unrounded to out_f32; the shards' partial sums add up to the layer output (an all-reduce when
+     the shards live on several GPUs).  expert_count == 0 means all E experts (the default). */
+  int32_t expert_lo, expert_count;
+  float* out_f32;               /* optional float [T, H]: the call's sum before rounding; `out` may then be NULL */
 } quads_moe_args;
 
 quads_status quads_moe_w4a4_rac(const quads_moe_args* args /* host */, void* cuda_stream);

@@ -34,6 +34,7 @@ class MoEArgs(C.Structure):
         ("h_bf16", _p), ("hq", _p), ("hsf", _p), ("r2q", _p), ("r2sf", _p), ("sel2", _p),
         ("workspace", _p), ("workspace_bytes", _sz),
         ("operand_mode", _i32), ("w13_bf16", _p),
+        ("expert_lo", _i32), ("expert_count", _i32), ("out_f32", _p),
     ]
 
 
@@ -193,7 +194,7 @@ def moe_workspace_bytes(T, H, I, E, topk, N=0):
 
 
 def moe_w4a4_rac(x, logits, w13, w2, topk, nsel13, nsel2, a2_gs, a13_gs=None, renormalize=True,
-                 export=False, workspace=None, out=None):
+                 export=False, workspace=None, out=None, expert_range=None, out_f32=None):
     """MoE layer forward.  w13 / w2: dicts with q [E,rows,K/2], sf (tiled, [E,bytes]), gs [E] as
     produced by fake_quant_weights(..., sf_layout=SF_TILED).  Returns dict(out=bf16 [T,H], ...)."""
     T, H = x.shape
@@ -209,9 +210,14 @@ def moe_w4a4_rac(x, logits, w13, w2, topk, nsel13, nsel2, a2_gs, a13_gs=None, re
     a.rac_nsel_13, a.rac_nsel_2 = nsel13, nsel2
     a.a13_gs, a.a2_gs = _ptr(a13_gs), _ptr(a2_gs)
     a.renormalize = 1 if renormalize else 0
+    if expert_range is not None:            # w13 / w2 hold the experts lo .. hi-1 only; out_f32 gets their partial sum
+        a.expert_lo, a.expert_count = expert_range[0], expert_range[1] - expert_range[0]
     res = {}
     res["out"] = out if out is not None else torch.empty(T, H, dtype=torch.bfloat16, device=dev)
     a.out = _ptr(res["out"])
+    if out_f32 is not None:
+        res["out_f32"] = out_f32
+        a.out_f32 = _ptr(out_f32)
     if export:
         u8, i32, f32 = torch.uint8, torch.int32, torch.float32
         res["ids"] = torch.empty(T, topk, dtype=i32, device=dev)

@@ -677,13 +677,19 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     if (!dense || a->operand_mode < QUADS_W4A16 || a->operand_mode > QUADS_W16A16 || a->rac_nsel_13 != 0)
       return QUADS_ERR_SHAPE;
   }
+  // expert-sharded execution: this call's experts
+  const int e_lo = (dense || a->expert_count == 0) ? 0 : a->expert_lo;
+  const int e_cnt = (dense || a->expert_count == 0) ? E : a->expert_count;
+  if (e_lo < 0 || e_cnt < 1 || e_lo + e_cnt > E) return QUADS_ERR_SHAPE;
+  if (dense && (a->expert_count != 0 || a->out_f32)) return QUADS_ERR_SHAPE;
   if (T == 0) return QUADS_OK;                      // nothing to do; x / out may be NULL
   if (a->operand_mode == QUADS_W16A4 || a->operand_mode == QUADS_W16A16) {
     if (!a->x || !a->w13_bf16 || !a->out) return QUADS_ERR_NULL;
     if (!aligned(a->w13_bf16, 16)) return QUADS_ERR_SHAPE;
-  } else if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || !a->out) {
+  } else if (!a->x || !a->w13_q || !a->w13_sf || !a->w13_gs || (!a->out && !a->out_f32)) {
     return QUADS_ERR_NULL;
   }
+  if (!aligned(a->out_f32, 16)) return QUADS_ERR_SHAPE;
   if (!dense && (!a->router_logits || !a->w2_q || !a->w2_sf || !a->w2_gs || !a->a2_gs)) return QUADS_ERR_NULL;
   if (!aligned(a->x, 32) || !aligned(a->w13_q, 16) || !aligned(a->w13_sf, 16) || !aligned(a->out, 16) ||
       (!dense && (!aligned(a->w2_q, 16) || !aligned(a->w2_sf, 16))))
@@ -774,12 +780,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     {
       auto route = E <= 32 ? route_kernel_t<1> : (E <= 64 ? route_kernel_t<2> : (E <= 128 ? route_kernel_t<4> : route_kernel_t<8>));
       QUADS_CUDA_OK(launch_kernel(route, dim3(L.n_chunks), dim3(256), (size_t)(0), rs, a->router_logits, T, E, topk,
-                                  a->renormalize, ids, wts, chunk_counts, expert_total, a->topk_ids, a->topk_w));
+                                  a->renormalize, ids, wts, chunk_counts, expert_total, a->topk_ids, a->topk_w, e_lo, e_lo + e_cnt));
     }
     trace_mark("route", st);
     QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(E), dim3(256), (size_t)(0), rs, E, L.n_chunks, cta_group, chunk_counts, expert_total, chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, a->expert_offsets));
     trace_mark("scan", st);
-    QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3(L.n_chunks), dim3(128), (size_t)(0), rs, T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
+    QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3(L.n_chunks), dim3(128), (size_t)(0), rs, T, E, topk, L.n_chunks, ids, wts, chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm, e_lo, e_lo + e_cnt));
   }
   trace_mark("permute", st);
 
@@ -878,12 +884,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   GemmMaps m1;
   if ((s = make_codes_map(&m1.a, P(L.xq_pad), pad_rows, H / 2, act_box)) != QUADS_OK) return s;
   if ((s = make_codes_map(&m1.r, P(L.rq_pad), pad_rows, H / 2, act_box)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&m1.b, a->w13_q, (uint64_t)E * N1, H / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m1.b, a->w13_q, (uint64_t)e_cnt * N1, H / 2)) != QUADS_OK) return s;
   if (cta_group == 2) {
     const uint64_t a_atoms = (uint64_t)(pad_rows / 128) * (H / 64);
     if ((s = make_sf_map(&m1.sfa, P(L.xsf), a_atoms)) != QUADS_OK) return s;
     if ((s = make_sf_map(&m1.sfr, P(L.rsf), a_atoms)) != QUADS_OK) return s;
-    if ((s = make_sf_map(&m1.sfb, a->w13_sf, (uint64_t)E * (quads_sf_tiled_bytes(N1, H) / 512))) != QUADS_OK) return s;
+    if ((s = make_sf_map(&m1.sfb, a->w13_sf, (uint64_t)e_cnt * (quads_sf_tiled_bytes(N1, H) / 512))) != QUADS_OK) return s;
   }
 
   GemmParams g{};
@@ -897,7 +903,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.tile_prefix = tile_prefix; g.offsets = offsets;
   g.status = header + kHdrStatus;
   g.b_rows_per_expert = N1;
-  g.n_experts = E;
+  g.n_experts = e_cnt;
+  g.expert_lo = e_lo;
   if (dense) {
     g.n_out = a->N;
     g.n_tiles_n = (a->N + 255) / 256;
@@ -935,7 +942,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   if (a->hq || a->hsf || a->r2q || a->r2sf) {
     const int64_t n = (int64_t)A * (I / 16);
-    QUADS_CUDA_OK(launch_kernel(export_site2_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), (size_t)(0), st, A, I, perm, pos_pad, P(L.hq_pad), P(L.hsf), P(L.r2q_pad), P(L.r2sf), mask2, a->hq, a->hsf, a->r2q, a->r2sf));
+    QUADS_CUDA_OK(launch_kernel(export_site2_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), (size_t)(0), st, A, header + kHdrAssignments, I, perm, pos_pad, P(L.hq_pad), P(L.hsf), P(L.r2q_pad), P(L.r2sf), mask2, a->hq, a->hsf, a->r2q, a->r2sf));
   }
 
   trace_mark("select2+mask", st);
@@ -944,12 +951,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   GemmMaps m2;
   if ((s = make_codes_map(&m2.a, P(L.hq_pad), pad_rows, I / 2, act_box)) != QUADS_OK) return s;
   if ((s = make_codes_map(&m2.r, P(L.r2q_pad), pad_rows, I / 2, act_box)) != QUADS_OK) return s;
-  if ((s = make_codes_map(&m2.b, a->w2_q, (uint64_t)E * H, I / 2)) != QUADS_OK) return s;
+  if ((s = make_codes_map(&m2.b, a->w2_q, (uint64_t)e_cnt * H, I / 2)) != QUADS_OK) return s;
   if (cta_group == 2) {
     const uint64_t a_atoms = (uint64_t)(pad_rows / 128) * (I / 64);
     if ((s = make_sf_map(&m2.sfa, P(L.hsf), a_atoms)) != QUADS_OK) return s;
     if ((s = make_sf_map(&m2.sfr, P(L.r2sf), a_atoms)) != QUADS_OK) return s;
-    if ((s = make_sf_map(&m2.sfb, a->w2_sf, (uint64_t)E * (quads_sf_tiled_bytes(H, I) / 512))) != QUADS_OK) return s;
+    if ((s = make_sf_map(&m2.sfb, a->w2_sf, (uint64_t)e_cnt * (quads_sf_tiled_bytes(H, I) / 512))) != QUADS_OK) return s;
   }
   GemmParams g2 = g;
   g2.K = I;
@@ -972,7 +979,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   }
   trace_mark("gemm2", st);
   const int64_t n8 = (int64_t)T * (H / 8);
-  QUADS_CUDA_OK(launch_kernel(combine_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), (size_t)(0), st, y_pad, pos_pad, wts, T, H, topk, static_cast<uint16_t*>(a->out)));
+  QUADS_CUDA_OK(launch_kernel(combine_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), (size_t)(0), st, y_pad, pos_pad, wts, T, H, topk, static_cast<uint16_t*>(a->out), a->out_f32));
   trace_mark("combine", st);
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
@@ -1087,12 +1094,12 @@ quads_status quads_moe_fp8_w8a8(const quads_moe_fp8_args* a, void* cuda_stream) 
   {
     auto route = E <= 32 ? route_kernel_t<1> : (E <= 64 ? route_kernel_t<2> : (E <= 128 ? route_kernel_t<4> : route_kernel_t<8>));
     QUADS_CUDA_OK(launch_kernel(route, dim3(L.n_chunks), dim3(256), (size_t)0, st, a->router_logits, T, E, topk, a->renormalize,
-                                ids, wts, chunk_counts, expert_total, a->topk_ids, (float*)nullptr));
+                                ids, wts, chunk_counts, expert_total, a->topk_ids, (float*)nullptr, 0, E));
   }
   QUADS_CUDA_OK(launch_kernel(scan_kernel, dim3(E), dim3(256), (size_t)0, st, E, L.n_chunks, 1, chunk_counts, expert_total,
                               chunk_base, offsets, tile_prefix, tile_expert, tile_rows, header, (int32_t*)nullptr));
   QUADS_CUDA_OK(launch_kernel(permute_kernel, dim3(L.n_chunks), dim3(128), (size_t)0, st, T, E, topk, L.n_chunks, ids, wts,
-                              chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm));
+                              chunk_base, offsets, tile_prefix, perm, pos_pad, row_token, row_weight, a->perm, 0, E));
   // ---- activation quantization (token order) and dispatch
   uint8_t* xq_tok = a->xq ? a->xq : P(L.xq_tok);
   uint8_t* xe_tok = a->xexp ? a->xexp : P(L.xe_tok);
@@ -1136,7 +1143,7 @@ quads_status quads_moe_fp8_w8a8(const quads_moe_fp8_args* a, void* cuda_stream) 
   }
   const int64_t n8 = (int64_t)T * (H / 8);
   QUADS_CUDA_OK(launch_kernel(combine_kernel, dim3((unsigned)((n8 + 255) / 256)), dim3(256), (size_t)0, st, g2.y_pad, pos_pad, wts,
-                              T, H, topk, static_cast<uint16_t*>(a->out)));
+                              T, H, topk, static_cast<uint16_t*>(a->out), (float*)nullptr));
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
 }

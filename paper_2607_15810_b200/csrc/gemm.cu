@@ -202,7 +202,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         const int mg = tile / p.n_tiles_n, nt = tile - mg * p.n_tiles_n;
         const int mt = mg * CG + (int)rank;
-        const int e = expert_of(mt);
+        const int e = expert_of(mt) - p.expert_lo;          // index into this call's weights
         const int brow0 = e * p.b_rows_per_expert + nt * (EPI == kEpiSwiGLU ? 128 : 256);
         const int brow1 = brow0 + p.half1_row_offset;
         const bool half1 = (EPI == kEpiSwiGLU) || (nt * 256 + 128 < p.n_out);
@@ -353,7 +353,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
       const int e = expert_of(mt);
       const bool valid = row_in_tile < rows_of(mt);
       const int prow = mt * kBM + row_in_tile;
-      const float scale = __fmul_rn(a_gs, gs_of(e));
+      const float scale = __fmul_rn(a_gs, gs_of(e - p.expert_lo));
       ok = mbar_wait(bar_tfull, (uint32_t)(it & 1), abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();

@@ -186,7 +186,7 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
     for (int item = blockIdx.x; item < total_items && ok; item += gridDim.x) {
       const int ch = item / n_ft, ft = item - ch * n_ft;
       const int mt = chunk_list[ch] >> 2, c = chunk_list[ch] & 3;
-      const int e = tab_expert[mt];
+      const int e = (int)tab_expert[mt] - p.expert_lo;                 // index into this call's weights
       const int wrow0 = e * p.b_rows_per_expert + ft * 128;            // gate rows (or the only rows)
       const int wrow1 = wrow0 + p.half1_row_offset;                   // up rows
       const int xrow = mt * 128 + c * kChunk;
@@ -321,7 +321,7 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
       const int n_pad = (n_rows + 15) & ~15;
       const int col0 = (c & 1) * kChunk;          // the chunk's first accumulator column
       const int row0 = mt * 128 + c * kChunk;     // padded dispatch row of the chunk's first token
-      const float scale = __fmul_rn(a_gs, tab_gs[e]);
+      const float scale = __fmul_rn(a_gs, tab_gs[e - p.expert_lo]);
       const int buf = it & 1;
       ok = mbar_wait(bar_tfull + 8 * buf, (uint32_t)((it >> 1) & 1), abort_flag, p.status);
       if (kDual) ok = epi_all(ok);               // also: the previous item's readers are done with hs / rs

@@ -57,8 +57,8 @@ __global__ void rac_dispatch_kernel(int H, int parts, const uint8_t* mask, const
                                     uint8_t* xsf_tiled, uint8_t* rq_pad, uint8_t* rsf_tiled);
 __global__ void mask_codes_kernel(uint8_t* codes, const int* n_rows_ptr, int C, const uint8_t* mask);
 __global__ void combine_kernel(const uint16_t* y_pad, const int32_t* pos_pad, const float* wts, int T, int H,
-                               int topk, uint16_t* out);
-__global__ void export_site2_kernel(int A, int I, const int32_t* perm, const int32_t* pos_pad,
+                               int topk, uint16_t* out, float* out_f32);
+__global__ void export_site2_kernel(int A, const int32_t* n_rows_ptr, int I, const int32_t* perm, const int32_t* pos_pad,
                                     const uint8_t* hq_pad, const uint8_t* hsf_tiled, const uint8_t* r2q_pad,
                                     const uint8_t* r2sf_tiled, const uint8_t* mask2, uint8_t* hq, uint8_t* hsf,
                                     uint8_t* r2q, uint8_t* r2sf);
@@ -70,14 +70,14 @@ __global__ void mismatch_norms_kernel(const uint16_t* a, const uint16_t* b, int6
 template <int NJ>
 __global__ void route_kernel_t(const float* logits, int T, int E, int topk, int renormalize, int32_t* ids,
                                float* wts, int32_t* chunk_counts, int32_t* expert_total, int32_t* ids_out,
-                               float* wts_out);
+                               float* wts_out, int e_lo, int e_hi);
 __global__ void scan_kernel(int E, int n_chunks, int tile_group, const int32_t* chunk_counts,
                             const int32_t* expert_total, int32_t* chunk_base, int32_t* offsets, int32_t* tile_prefix,
                             int32_t* tile_expert, int32_t* tile_rows, int32_t* header, int32_t* offsets_out);
 __global__ void permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* ids, const float* wts,
                                const int32_t* chunk_base, const int32_t* offsets, const int32_t* tile_prefix,
                                int32_t* perm, int32_t* pos_pad, int32_t* row_token, float* row_weight,
-                               int32_t* perm_out);
+                               int32_t* perm_out, int e_lo, int e_hi);
 __global__ void dense_dispatch_kernel(int T, int tile_group, int32_t* pos_pad, int32_t* row_token, float* row_weight,
                                       int32_t* tile_expert, int32_t* tile_rows, int32_t* header);
 
@@ -96,7 +96,8 @@ struct GemmParams {
   int b_rows_per_expert; // weight rows per expert
   int half1_row_offset;  // weight-row distance from the tile's first half to its second half
   int has_resid;         // 1: also accumulate the (negated, masked) residual operand
-  int n_experts;         // entries of b_gs
+  int n_experts;         // entries of b_gs (the experts whose weights this call holds)
+  int expert_lo;         // global id of the first of them: weights / scales are indexed by (expert - expert_lo)
   const int32_t* header;
   const int32_t* tile_expert;
   const int32_t* tile_rows;

@@ -1125,7 +1125,8 @@ mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_pt
 // One thread per (token, 8 columns).
 __global__ void __launch_bounds__(256)
 combine_kernel(const uint16_t* __restrict__ y_pad, const int32_t* __restrict__ pos_pad,
-               const float* __restrict__ wts, int T, int H, int topk, uint16_t* __restrict__ out) {
+               const float* __restrict__ wts, int T, int H, int topk, uint16_t* __restrict__ out,
+               float* __restrict__ out_f32) {
   pdl_sync();
   const int per_row = H >> 3;
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -1158,15 +1159,22 @@ combine_kernel(const uint16_t* __restrict__ y_pad, const int32_t* __restrict__ p
       for (int k = 0; k < 8; ++k) acc[k] = __fmaf_rn(w[j], f[k], acc[k]);
     }
   }
-  reinterpret_cast<uint4*>(out + (size_t)t * H)[c] =
-      make_uint4(f32x2_to_bf16x2(acc[0], acc[1]), f32x2_to_bf16x2(acc[2], acc[3]),
-                 f32x2_to_bf16x2(acc[4], acc[5]), f32x2_to_bf16x2(acc[6], acc[7]));
+  if (out_f32) {                                       // partial sums of an expert-sharded call, unrounded
+    float4* d = reinterpret_cast<float4*>(out_f32 + (size_t)t * H) + 2 * c;
+    d[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    d[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+  }
+  if (out)
+    reinterpret_cast<uint4*>(out + (size_t)t * H)[c] =
+        make_uint4(f32x2_to_bf16x2(acc[0], acc[1]), f32x2_to_bf16x2(acc[2], acc[3]),
+                   f32x2_to_bf16x2(acc[4], acc[5]), f32x2_to_bf16x2(acc[6], acc[7]));
 }
 
 // Export of padded dispatch-order buffers into linear dispatch order.
 // One thread per (dispatched row, 16-channel block).
 __global__ void __launch_bounds__(256)
-export_site2_kernel(int A, int I, const int32_t* __restrict__ perm, const int32_t* __restrict__ pos_pad,
+export_site2_kernel(int A, const int32_t* __restrict__ n_rows_ptr, int I, const int32_t* __restrict__ perm,
+                    const int32_t* __restrict__ pos_pad,
                     const uint8_t* __restrict__ hq_pad, const uint8_t* __restrict__ hsf_tiled,
                     const uint8_t* __restrict__ r2q_pad, const uint8_t* __restrict__ r2sf_tiled,
                     const uint8_t* __restrict__ mask2, uint8_t* __restrict__ hq, uint8_t* __restrict__ hsf, uint8_t* __restrict__ r2q,
@@ -1176,6 +1184,7 @@ export_site2_kernel(int A, int I, const int32_t* __restrict__ perm, const int32_
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (int64_t)A * k16) return;
   const int row = (int)(i / k16), kb = (int)(i - (int64_t)row * k16);
+  if (row >= *n_rows_ptr) return;          // an expert-sharded call dispatches only its own experts' rows
   const int p = pos_pad[perm[row]];
   const size_t so = sf_tiled_offset(p, kb, I >> 6);
   if (hq) *reinterpret_cast<uint2*>(hq + (size_t)row * (I >> 1) + kb * 8) =

@@ -23,7 +23,8 @@ template <int NJ>
 __global__ void __launch_bounds__(256)
 route_kernel_t(const float* __restrict__ logits, int T, int E, int topk, int renormalize,
              int32_t* __restrict__ ids, float* __restrict__ wts, int32_t* __restrict__ chunk_counts,
-             int32_t* __restrict__ expert_total, int32_t* __restrict__ ids_out, float* __restrict__ wts_out) {
+             int32_t* __restrict__ expert_total, int32_t* __restrict__ ids_out, float* __restrict__ wts_out,
+             int e_lo, int e_hi) {
   pdl_sync();
   __shared__ int hist[kMaxExperts];
   for (int i = threadIdx.x; i < E; i += blockDim.x) hist[i] = 0;
@@ -108,7 +109,7 @@ route_kernel_t(const float* __restrict__ logits, int T, int E, int topk, int ren
       wts[(size_t)t * topk + lane] = w;
       if (ids_out) ids_out[(size_t)t * topk + lane] = my_id[a];
       if (wts_out) wts_out[(size_t)t * topk + lane] = w;
-      atomicAdd(&hist[my_id[a]], 1);
+      if (my_id[a] >= e_lo && my_id[a] < e_hi) atomicAdd(&hist[my_id[a]], 1);   // only this call's experts get rows
     }
   }
   __syncthreads();
@@ -118,10 +119,10 @@ route_kernel_t(const float* __restrict__ logits, int T, int E, int topk, int ren
   }
 }
 
-template __global__ void route_kernel_t<1>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
-template __global__ void route_kernel_t<2>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
-template __global__ void route_kernel_t<4>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
-template __global__ void route_kernel_t<8>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*);
+template __global__ void route_kernel_t<1>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*, int, int);
+template __global__ void route_kernel_t<2>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*, int, int);
+template __global__ void route_kernel_t<4>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*, int, int);
+template __global__ void route_kernel_t<8>(const float*, int, int, int, int, int32_t*, float*, int32_t*, int32_t*, int32_t*, float*, int, int);
 
 // One CTA per expert, 256 threads.  From the experts' totals: the exclusive scan over experts of
 // counts (offsets) and of 128-row tile counts (tile_prefix; every expert gets a multiple of
@@ -209,7 +210,8 @@ __global__ void __launch_bounds__(128)
 permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__ ids, const float* __restrict__ wts,
                const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ offsets,
                const int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ pos_pad,
-               int32_t* __restrict__ row_token, float* __restrict__ row_weight, int32_t* __restrict__ perm_out) {
+               int32_t* __restrict__ row_token, float* __restrict__ row_weight, int32_t* __restrict__ perm_out,
+               int e_lo, int e_hi) {
   pdl_sync();
   __shared__ int run[4][kMaxExperts];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -223,8 +225,9 @@ permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__
   // pass 1: this warp's count per expert
   for (int i0 = i_begin; i0 < i_end; i0 += 32) {
     const int i = i0 + lane;
-    const bool active = i < i_end;
-    const int e = active ? ids[t0 * topk + i] : (0x40000000 + lane);
+    int e = i < i_end ? ids[t0 * topk + i] : -1;
+    const bool active = e >= e_lo && e < e_hi;              // an assignment to an expert of this call
+    if (!active) e = 0x40000000 + lane;
     const unsigned same = __match_any_sync(0xFFFFFFFFu, e);
     if (active && (same & ((1u << lane) - 1u)) == 0) run[warp][e] += __popc(same);
     __syncwarp();
@@ -244,9 +247,11 @@ permute_kernel(int T, int E, int topk, int n_chunks, const int32_t* __restrict__
   // pass 2: hand out the rows
   for (int i0 = i_begin; i0 < i_end; i0 += 32) {
     const int i = i0 + lane;
-    const bool active = i < i_end;
     const int flat = t0 * topk + i;
-    const int e = active ? ids[flat] : (0x40000000 + lane);
+    int e = i < i_end ? ids[flat] : -1;
+    const bool active = e >= e_lo && e < e_hi;
+    if (i < i_end && !active) pos_pad[flat] = -1;           // another call's expert (expert-sharded execution)
+    if (!active) e = 0x40000000 + lane;
     const unsigned same = __match_any_sync(0xFFFFFFFFu, e);
     const int rank = __popc(same & ((1u << lane) - 1u));
     int base = 0;

@@ -18,9 +18,11 @@
 // tenth faster, but every expert's rows must then be padded to a multiple of 256).
 // Every CTA loads what it needs itself; no load is shared across the cluster.
 //
-// One persistent CTA per SM, 18 warps:
-//   warp 0     producer: TMA tile loads of packed FP4 (128-byte swizzle) and bulk
-//              copies of 512-byte scale atoms into a 3-stage shared-memory ring;
+// One persistent CTA per SM, 19 warps:
+//   warp 0     producer: TMA tile loads of packed FP4 (128-byte swizzle) into a 3-stage
+//              shared-memory ring;
+//   warp 18    second producer: the bulk copies of the stage's 512-byte scale atoms (in the
+//              CTA-pair variant warp 0 issues those too, as TMA boxes, and this warp idles);
 //   warp 1     tensor-memory allocation; one thread copies scale atoms to TMEM
 //              (tcgen05.cp) and issues the MMAs, releasing stages with
 //              tcgen05.commit;
@@ -46,7 +48,7 @@ constexpr int kSfA = kKSteps * 512;               // one atom (128 rows x 4 bloc
 constexpr int kSfB = 2 * kSfA;                    // scales of all 256 weight rows
 constexpr int kOffR = kTileA;
 constexpr int kOffB = 2 * kTileA;
-constexpr int kThreads = 576;
+constexpr int kThreads = 608;
 constexpr int kEpiWarps = 16;
 constexpr int kTmemCols = 512;
 constexpr int kMaxTableTiles = 2048;               // M-tiles whose expert / row count fit the shared-memory tables
@@ -191,8 +193,14 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
   const bool resid = p.has_resid != 0;
   const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ producer (whole warp, one lane issues)
+  // Two loading warps share a stage's copies: warp 0 the operand tiles (and the byte count), warp 18
+  // the scale atoms (single-CTA variant; an asynchronous copy costs its issuing thread tens of
+  // nanoseconds whatever its size: first projection 195 -> 193 us, second 116 -> 113.5 us).  All
+  // copies of a stage credit the same barrier.
+  const int load_role = warp == 0 ? 0 : (warp == 18 ? 1 : -1);
+  if (load_role >= 0) {
+    // ------------------------------------------------------------ producers (whole warp, one lane issues)
+    if (CG == 1 || load_role == 0)                  // (the pair variant keeps one loading warp; warp 18 idles there)
     {
       const bool issuer = elect_one();
       uint32_t stage = 0, phase = 0;
@@ -228,15 +236,20 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
           const size_t sf_off = (size_t)ks * (size_t)kSfA;
           if (issuer) {
             if (CG == 1) {
-              mbar_expect_tx(full, data_bytes + sf_bytes * sf_count);
-              tma_load_2d(sbase, tm_a, kc, mt * kBM, full);
-              if (resid) tma_load_2d(sbase + kOffR, tm_r, kc, mt * kBM, full);
-              tma_load_2d(sbase + kOffB, tm_b, kc, brow0, full);
-              if (half1) tma_load_2d(sbase + kOffB + kTileA, tm_b, kc, brow1, full);
-              bulk_load(sbase + C::kOffSfA, asf + sf_off, sf_bytes, full);
-              if (resid) bulk_load(sbase + C::kOffSfR, rsf + sf_off, sf_bytes, full);
-              bulk_load(sbase + C::kOffSfB, bsf0 + sf_off, sf_bytes, full);
-              if (half1) bulk_load(sbase + C::kOffSfB + kSfA, bsf1 + sf_off, sf_bytes, full);
+              const bool do_tiles = load_role == 0, do_sf = load_role == 1;
+              if (do_tiles) {
+                mbar_expect_tx(full, data_bytes + sf_bytes * sf_count);
+                tma_load_2d(sbase, tm_a, kc, mt * kBM, full);
+                if (resid) tma_load_2d(sbase + kOffR, tm_r, kc, mt * kBM, full);
+                tma_load_2d(sbase + kOffB, tm_b, kc, brow0, full);
+                if (half1) tma_load_2d(sbase + kOffB + kTileA, tm_b, kc, brow1, full);
+              }
+              if (do_sf) {
+                bulk_load(sbase + C::kOffSfA, asf + sf_off, sf_bytes, full);
+                if (resid) bulk_load(sbase + C::kOffSfR, rsf + sf_off, sf_bytes, full);
+                bulk_load(sbase + C::kOffSfB, bsf0 + sf_off, sf_bytes, full);
+                if (half1) bulk_load(sbase + C::kOffSfB + kSfA, bsf1 + sf_off, sf_bytes, full);
+              }
             } else {
               // every load of either CTA credits the LEADER's barrier; scale atoms travel as TMA
               // boxes (kKSteps atoms of 512 bytes; a K tail reads, and counts, the full box)

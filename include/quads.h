@@ -398,10 +398,9 @@ size_t quads_mismatch_norms_workspace_bytes(void);
  *   mode 1  two MMAs + four scale copies per step (first projection with RAC);
  *   mode 2  one MMA + three scale copies (plain W4A4);
  *   mode 3  two MMAs, no copies;  mode 4  as mode 1 with the copies issued by a
- *   second thread.
+ *   second thread;  mode 5  one 128 x 128 x 64 MMA.
  * Time it with events on `cuda_stream`; *flop_out (host, may be NULL) receives
- * the floating-point operations of the launch (2 * 128 * 256 * 64 per MMA and
- * SM).  Scale bytes in `operands` should avoid the NaN code 0x7F.  The wait for
+ * the floating-point operations of the launch (2 * M * N * 64 per MMA and SM).  Scale bytes in `operands` should avoid the NaN code 0x7F.  The wait for
  * the pipe to drain is bounded; a give-up writes QUADS_ERR_TIMEOUT to
  * *status_word (device int32, zero it first).
  */

@@ -11,6 +11,8 @@
 //   mode 2   one MMA + three scale copies per step                      (plain W4A4)
 //   mode 3   two MMAs per step, scales copied once                      (RAC without its copies)
 //   mode 4   as mode 1, but the copies are issued by a second warp      (two issuing threads)
+//   mode 5   one N = 128 MMA (128 x 128 x 64) per step, scales copied once
+// (M is 128 for every block-scaled kind with cta_group::1: there is no half-height form to probe.)
 // Results in tensor memory are never read; every wait is bounded.
 #include "kernels.cuh"
 #include "tcgen05.cuh"
@@ -68,6 +70,7 @@ fp4_pipe_probe_kernel(const uint8_t* __restrict__ operands, int mode, int k_step
     tc_cp_sf<1>(c + 32 + 8 * j + 4, ((uint64_t)kSfHi << 32) | (sfb_lo + 128 + 32 * j));
   };
   const bool two_mma = mode == 1 || mode == 3 || mode == 4;
+  const uint32_t idesc_m = mode == 5 ? ((1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24)) : idesc;
   const bool copies = mode == 1 || mode == 2;
   if (warp == 1) {
     const bool issuer = elect_one();
@@ -78,7 +81,7 @@ fp4_pipe_probe_kernel(const uint8_t* __restrict__ operands, int mode, int k_step
         if (copies) copy_sf(j, buf, two_mma);
         const uint32_t c = sfcol + buf * 64;
         const uint64_t bdesc = ((uint64_t)kSwHi << 32) | (b_lo + 2 * j);
-        tc_mma_nvf4<1>(tmem, ((uint64_t)kSwHi << 32) | (a_lo + 2 * j), bdesc, idesc, c + 4 * j, c + 32 + 8 * j,
+        tc_mma_nvf4<1>(tmem, ((uint64_t)kSwHi << 32) | (a_lo + 2 * j), bdesc, idesc_m, c + 4 * j, c + 32 + 8 * j,
                        s > 0 ? 1u : 0u);
         if (two_mma)
           tc_mma_nvf4<1>(tmem, ((uint64_t)kSwHi << 32) | (r_lo + 2 * j), bdesc, idesc, c + 16 + 4 * j, c + 32 + 8 * j, 1u);
@@ -112,7 +115,7 @@ using namespace quads;
 extern "C" quads_status quads_fp4_pipe_probe(int32_t mode, int32_t k_steps, const void* operands, size_t operand_bytes,
                                              int32_t* status_word, double* flop_out, void* cuda_stream) {
   g_launch_count = 0;
-  if (mode < 0 || mode > 4 || k_steps < 1) return QUADS_ERR_SHAPE;
+  if (mode < 0 || mode > 5 || k_steps < 1) return QUADS_ERR_SHAPE;
   if (!operands || !status_word) return QUADS_ERR_NULL;
   if (operand_bytes < (size_t)kPStageBytes || (reinterpret_cast<uintptr_t>(operands) & 15)) return QUADS_ERR_WORKSPACE;
   int dev = 0, sms = 0, cc = 0;
@@ -126,7 +129,8 @@ extern "C" quads_status quads_fp4_pipe_probe(int32_t mode, int32_t k_steps, cons
   note_launch();
   QUADS_CUDA_OK(cudaGetLastError());
   const int mmas = (mode == 1 || mode == 3 || mode == 4) ? 2 : 1;
-  if (flop_out) *flop_out = (double)sms * (double)k_steps * mmas * 2.0 * 128.0 * 256.0 * 64.0;
+  const double shape = mode == 5 ? 128.0 * 128.0 : 128.0 * 256.0;
+  if (flop_out) *flop_out = (double)sms * (double)k_steps * mmas * 2.0 * shape * 64.0;
   return QUADS_OK;
 }
 

@@ -738,7 +738,35 @@ def run_ours(args):
             tt = timed(fn_, 20)
             cmp_ms[name_] = sum(tt) / len(tt)
         assert B.moe_async_status(fws) == 0
+        # how well each arm's first projection uses its own tensor-core peak (FP8 = 2 x, FP4 = 4 x the measured bf16 rate):
+        # the FP8 kernels here are single-CTA 128 x 256 tiles, which need twice the bytes per MMA cycle of the FP4 ones
+        B.moe_set_kernel_timing(True)
+        kt = {}
+        for name_, fn_ in (("fp8_w8a8", fp8_step), ("nvfp4_plain", plain_step)):
+            acc_ = []
+            for _ in range(5):
+                flush_l2()
+                fn_()
+                acc_.append(B.moe_last_kernel_ms())
+            kt[name_] = [sum(v[i] for v in acc_) / len(acc_) for i in (0, 1)]
+        B.moe_set_kernel_timing(False)
+        f1_plain = 2.0 * A * H * 2 * I
+        f2_plain = 2.0 * A * I * H
+        fp8_peak = 2.0 * peaks["bf16_tflops"]
+        # the FP8 layer if its two GEMMs ran at the fraction of the FP8 peak that the plain-W4A4 GEMMs reach of the FP4 peak
+        eq1 = f1_plain / (f1_plain / (kt["nvfp4_plain"][0] * 1e-3) / fp4_peak * fp8_peak) * 1e3
+        eq2 = f2_plain / (f2_plain / (kt["nvfp4_plain"][1] * 1e-3) / fp4_peak * fp8_peak) * 1e3
+        fp8_equal_ms = cmp_ms["fp8_w8a8"] - kt["fp8_w8a8"][0] - kt["fp8_w8a8"][1] + eq1 + eq2
         aux["fp8_comparison_%s" % shape.name] = {
+            "fp8_ms_at_equal_gemm_efficiency": fp8_equal_ms,
+            "ratios_at_equal_gemm_efficiency": {"plain_w4a4_over_fp8": fp8_equal_ms / cmp_ms["nvfp4_plain"],
+                                                "rac_w13_over_fp8": fp8_equal_ms / cmp_ms["nvfp4_rac_w13"],
+                                                "rac_both_over_fp8": fp8_equal_ms / cmp_ms["nvfp4_rac_both"]},
+            "gemm_ms": kt,
+            "gemm1_frac_of_own_peak": {"fp8_w8a8": f1_plain / (kt["fp8_w8a8"][0] * 1e-3) / 1e12 / (2.0 * peaks["bf16_tflops"]),
+                                       "nvfp4_plain": f1_plain / (kt["nvfp4_plain"][0] * 1e-3) / 1e12 / fp4_peak},
+            "caveat": "the FP8 GEMMs of this repository are less tuned than the FP4 ones (see gemm1_frac_of_own_peak): the "
+                      "ratios below overstate what a tuned FP8 kernel would leave, most of all at prefill",
             "ms_per_layer": cmp_ms,
             "plain_w4a4_over_fp8": cmp_ms["fp8_w8a8"] / cmp_ms["nvfp4_plain"],
             "rac_w13_over_fp8": cmp_ms["fp8_w8a8"] / cmp_ms["nvfp4_rac_w13"],

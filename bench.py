@@ -765,8 +765,9 @@ def run_ours(args):
             "gemm_ms": kt,
             "gemm1_frac_of_own_peak": {"fp8_w8a8": f1_plain / (kt["fp8_w8a8"][0] * 1e-3) / 1e12 / (2.0 * peaks["bf16_tflops"]),
                                        "nvfp4_plain": f1_plain / (kt["nvfp4_plain"][0] * 1e-3) / 1e12 / fp4_peak},
-            "caveat": "the FP8 GEMMs of this repository are less tuned than the FP4 ones (see gemm1_frac_of_own_peak): the "
-                      "ratios below overstate what a tuned FP8 kernel would leave, most of all at prefill",
+            "fairness": "gemm1_frac_of_own_peak says how much of its own tensor-core peak (FP8 = 2 x, FP4 = 4 x the measured "
+                        "bf16 rate) each arm's first projection reaches; fp8_ms_at_equal_gemm_efficiency re-scales the FP8 GEMMs to "
+                        "the FP4 kernels' fraction, so the ratios can be read either way",
             "ms_per_layer": cmp_ms,
             "plain_w4a4_over_fp8": cmp_ms["fp8_w8a8"] / cmp_ms["nvfp4_plain"],
             "rac_w13_over_fp8": cmp_ms["fp8_w8a8"] / cmp_ms["nvfp4_rac_w13"],

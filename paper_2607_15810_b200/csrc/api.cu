@@ -214,7 +214,7 @@ inline void trace_mark(const char* name, cudaStream_t st) {
 // activation chain (amax -> quantize -> select); both are joined before the dispatch copy.
 struct SideStream {
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, mid = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, mid = nullptr, tables = nullptr, join = nullptr;
   bool ok = false;
 };
 std::mutex g_side_mu;
@@ -230,6 +230,7 @@ SideStream* side_stream() {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.mid, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.tables, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s.ok = true;
   }
@@ -841,7 +842,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   trace_mark("rac_stats", st);
   // The dispatched copies of Q(x) need only the dispatch order and the codes: with a side stream
   // they are written there, next to the channel selection; the residual copies (which need the
-  // selection) follow on the main stream.
+  // selection and the dispatch tables, not the other copies) follow on the main stream and may run
+  // beside them: the two streams meet again only in front of the first projection.
   const bool split_scatter = side != nullptr && nsel13 > 0;
   auto dispatch = [&](int parts, cudaStream_t s_) {
     return launch_kernel(rac_dispatch_kernel, dim3(L.m_tiles_max), dim3(256), (size_t)(0), s_, H, parts, mask13, header,
@@ -850,6 +852,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   };
   if (side) {
     if (split_scatter) {
+      QUADS_CUDA_OK(cudaEventRecord(side->tables, side->stream));      // routing tables complete
       QUADS_CUDA_OK(cudaEventRecord(side->mid, st));
       QUADS_CUDA_OK(cudaStreamWaitEvent(side->stream, side->mid, 0));
       QUADS_CUDA_OK(dispatch(1, side->stream));
@@ -862,7 +865,9 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     if (s != QUADS_OK) return s;
   }
   trace_mark("select13", st);
-  if (side) {
+  if (split_scatter) {
+    QUADS_CUDA_OK(cudaStreamWaitEvent(st, side->tables, 0));
+  } else if (side) {
     side_guard.join();
     side_lock.unlock();
   }
@@ -874,6 +879,10 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
       const int64_t chunks = (int64_t)T * (H / 32);
       QUADS_CUDA_OK(launch_kernel(rac_scatter_kernel, dim3((unsigned)((chunks + 255) / 256)), dim3(256), (size_t)(0), st, T, H, 2, mask13, 0, pos_pad, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad), P(L.xsf), P(L.rq_pad), P(L.rsf), a->rq, a->rsf));
     }
+  }
+  if (split_scatter) {
+    side_guard.join();
+    side_lock.unlock();
   }
   trace_mark("rac_dispatch", st);
   // ---- tensor maps

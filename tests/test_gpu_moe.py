@@ -2,6 +2,7 @@
 config, small MoE layers compared in full, and the decode / prefill / large
 configs at full size."""
 import os
+import random
 import sys
 
 import numpy as np
@@ -189,6 +190,27 @@ EDGE_SHAPES = [
 @pytest.mark.parametrize("shape", EDGE_SHAPES, ids=[s.name for s in EDGE_SHAPES])
 def test_moe_edge_shapes(B, shape):
     _moe_small(B, None, 0.5, 0.5, True, shape=shape)
+
+
+def _random_shape(seed):
+    rng = random.Random(seed)
+    E = rng.choice([1, 2, 3, 5, 8, 16, 24, 32, 64])
+    topk = rng.randint(1, min(E, 8))
+    T = rng.choice([1, 2, 7, 31, 64, 129, 200, 257, 400, 777])
+    H = 128 * rng.choice([1, 2, 3, 4, 5, 8])
+    I = 128 * rng.choice([1, 2, 3, 4])
+    hot = min(rng.choice([0, 0, 1, 2]), E)
+    sh = synth.MoEShape("random%d" % seed, 1000 + seed, T, H, E, topk, I, 0.05, rng.randint(0, 4), 3.0, 10.0,
+                        hot, 0.5 if hot else 0.0)
+    return sh, rng.choice([0.0, 0.25, 0.5, 1.0]), rng.choice([0.0, 0.5, 1.0]), rng.random() < 0.5
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_moe_random_shapes(B, seed):
+    """Seeded random layer shapes, expert counts, top-k, hot experts, compensation ratios: the whole layer
+    against the oracle as in the named cases above."""
+    sh, f13, f2, renorm = _random_shape(seed)
+    _moe_small(B, None, f13, f2, renorm, shape=sh)
 
 
 def test_zero_tokens_is_a_no_op(B):

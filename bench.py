@@ -868,6 +868,48 @@ def run_ours(args):
             aux["decode_48_layers_note"] = ("%d MoE layers x %.0f MB of weights, T=%d, static activation scales, one graph "
                                             "replay per step") % (n_layers, wbytes / 1e6, dsh.T)
             del layers
+            # the large layer (T=4096, H=4096, I=1536, 128 experts, ~256 rows per expert: the size
+            # where weight streaming and the tensor pipe are about level), weights drawn on the device
+            lsh = synth.MOE_SHAPES["large"]
+            gl = torch.Generator(device=dev)
+            gl.manual_seed(lsh.seed)
+
+            def pack_large(rows, cols):
+                parts = []
+                for e0 in range(0, lsh.E, 16):
+                    w = (torch.randn(16, rows, cols, generator=gl, device=dev) * lsh.w_std).to(torch.bfloat16)
+                    parts.append(B.fake_quant_weights(w, want_fq=False, sf_layout=B.SF_TILED))
+                    del w
+                return {k: torch.cat([p[k] for p in parts]) for k in ("q", "sf", "gs")}
+            l13, l2 = pack_large(2 * lsh.I, lsh.H), pack_large(lsh.H, lsh.I)
+            lx, _ = synth.activations(lsh)
+            llg = synth.router_logits(lsh)
+            lx, llg = lx.to(dev), llg.to(dev)
+            la2 = torch.tensor([synth.H_GLOBAL_SCALE[lsh.name]], dtype=torch.float32, device=dev)
+            lws = torch.empty(B.moe_workspace_bytes(lsh.T, lsh.H, lsh.I, lsh.E, lsh.topk), dtype=torch.uint8, device=dev)
+            lout = torch.empty(lsh.T, lsh.H, dtype=torch.bfloat16, device=dev)
+            large = {}
+            for vname, (v13, v2) in (("rac_both", (lsh.H // 2, lsh.I // 2)), ("rac_w13", (lsh.H // 2, 0)), ("plain", (0, 0))):
+                def lstep(v13=v13, v2=v2):
+                    B.moe_w4a4_rac(lx, llg, l13, l2, lsh.topk, v13, v2, la2, workspace=lws, out=lout)
+                for _ in range(3):
+                    flush_l2()
+                    lstep()
+                tl = timed(lstep, 20)
+                lms = sum(tl) / len(tl)
+                A_l = lsh.T * lsh.topk
+                f_alg = 6.0 * A_l * lsh.H * lsh.I * (1.0 + (2.0 / 3.0) * v13 / lsh.H + (1.0 / 3.0) * v2 / lsh.I)
+                large[vname] = {"ms_per_step": lms, "tokens_per_s": lsh.T / (lms * 1e-3),
+                                "algorithmic_tflops": f_alg / (lms * 1e-3) / 1e12,
+                                "frac_of_fp4_peak": f_alg / (lms * 1e-3) / 1e12 / fp4_peak}
+            assert B.moe_async_status(lws) == 0
+            lbytes = sum(t.numel() * t.element_size() for g_ in (l13, l2) for t in g_.values())
+            large["weight_bytes"] = lbytes
+            large["weight_stream_floor_ms"] = lbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+            large["note"] = ("T=%d, H=%d, I=%d, E=%d, top-%d; cold weights, L2 flushed between steps; weights N(0, %.3f) "
+                             "drawn on the device" % (lsh.T, lsh.H, lsh.I, lsh.E, lsh.topk, lsh.w_std))
+            aux["large_layer"] = large
+            del l13, l2, lws
         line["aux"] = aux
 
     if world == 1 and not args.no_cpu_baseline:

@@ -846,7 +846,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   // beside them: the two streams meet again only in front of the first projection.
   const bool split_scatter = side != nullptr && nsel13 > 0;
   auto dispatch = [&](int parts, cudaStream_t s_) {
-    return launch_kernel(rac_dispatch_kernel, dim3(L.m_tiles_max), dim3(256), (size_t)(0), s_, H, parts, mask13, header,
+    auto k = parts == 1 ? rac_dispatch_kernel<1> : (parts == 2 ? rac_dispatch_kernel<2> : rac_dispatch_kernel<3>);
+    return launch_kernel(k, dim3(L.m_tiles_max), dim3(256), (size_t)(0), s_, H, mask13, header,
                          tile_rows, row_token, P(L.xq_tok), P(L.xsf_tok), P(L.rq_tok), P(L.rsf_tok), P(L.xq_pad),
                          P(L.xsf), P(L.rq_pad), P(L.rsf));
   };

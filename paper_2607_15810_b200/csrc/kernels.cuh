@@ -51,7 +51,8 @@ __global__ void rac_scatter_kernel(int T, int H, int parts, const uint8_t* mask,
                                    const int32_t* pos_pad, const uint8_t* xq, const uint8_t* xsf, const uint8_t* rq,
                                    const uint8_t* rsf, uint8_t* xq_pad, uint8_t* xsf_tiled, uint8_t* rq_pad,
                                    uint8_t* rsf_tiled, uint8_t* rq_exp, uint8_t* rsf_exp);
-__global__ void rac_dispatch_kernel(int H, int parts, const uint8_t* mask, const int32_t* header,
+template <int kParts>   // bit 0: copies of Q(x), bit 1: masked, negated copies of the residual
+__global__ void rac_dispatch_kernel(int H, const uint8_t* mask, const int32_t* header,
                                     const int32_t* tile_rows, const int32_t* row_token, const uint8_t* xq,
                                     const uint8_t* xsf, const uint8_t* rq, const uint8_t* rsf, uint8_t* xq_pad,
                                     uint8_t* xsf_tiled, uint8_t* rq_pad, uint8_t* rsf_tiled);

@@ -983,8 +983,10 @@ rac_scatter_kernel(int T, int H, int parts, const uint8_t* __restrict__ mask, in
 // grid = upper bound of the tile count (tiles beyond header[kHdrMTiles] leave at once), 256 threads.
 // ---------------------------------------------------------------------------
 constexpr int kDispatchSlab = 32;                   // scale atoms (K = 64 each) staged per pass
-__global__ void __launch_bounds__(256)
-rac_dispatch_kernel(int H, int parts, const uint8_t* __restrict__ mask, const int32_t* __restrict__ header,
+constexpr int kDispatchRows = 8;                    // rows (16-byte loads) in flight per thread (4: 2 us slower per half, 16: spills)
+template <int kParts>
+__global__ void __launch_bounds__(256, 4)
+rac_dispatch_kernel(int H, const uint8_t* __restrict__ mask, const int32_t* __restrict__ header,
                     const int32_t* __restrict__ tile_rows, const int32_t* __restrict__ row_token,
                     const uint8_t* __restrict__ xq, const uint8_t* __restrict__ xsf, const uint8_t* __restrict__ rq,
                     const uint8_t* __restrict__ rsf, uint8_t* __restrict__ xq_pad, uint8_t* __restrict__ xsf_tiled,
@@ -994,10 +996,11 @@ rac_dispatch_kernel(int H, int parts, const uint8_t* __restrict__ mask, const in
   if (mt >= header[kHdrMTiles]) return;
   const int n_rows = tile_rows[mt];
   __shared__ int tok[128];
-  __shared__ __align__(16) uint8_t atoms[2][kDispatchSlab * 512];
+  __shared__ __align__(16) uint8_t atoms[kParts == 3 ? 2 : 1][kDispatchSlab * 512];
   if (threadIdx.x < 128) tok[threadIdx.x] = threadIdx.x < n_rows ? row_token[mt * 128 + threadIdx.x] : -1;
   __syncthreads();
-  const bool do_x = (parts & 1) != 0, do_r = (parts & 2) != 0;
+  constexpr bool do_x = (kParts & 1) != 0, do_r = (kParts & 2) != 0;
+  constexpr int kRows = kParts == 3 ? kDispatchRows / 2 : kDispatchRows;   // the same number of loads in flight
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int per_row = H >> 5;                         // 16-byte chunks of codes per row
   const size_t row_bytes = (size_t)(H >> 1);
@@ -1008,25 +1011,25 @@ rac_dispatch_kernel(int H, int parts, const uint8_t* __restrict__ mask, const in
       const uint8_t* m = mask + c * 32;
       m0 = nibble_mask8(m); m1 = nibble_mask8(m + 8); m2 = nibble_mask8(m + 16); m3 = nibble_mask8(m + 24);
     }
-    for (int r0 = warp; r0 < n_rows; r0 += 32) {      // four rows in flight per thread
-      uint4 xv[4], rv[4];
+    for (int r0 = warp; r0 < n_rows; r0 += 8 * kRows) {   // kRows rows in flight per thread
+      uint4 xv[do_x ? kRows : 1], rv[do_r ? kRows : 1];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < kRows; ++j) {
         const int r = r0 + 8 * j;
         if (r < n_rows) {
           const size_t so = (size_t)tok[r] * row_bytes + (size_t)c * 16;
-          if (do_x) xv[j] = __ldg(reinterpret_cast<const uint4*>(xq + so));
-          if (do_r) rv[j] = __ldg(reinterpret_cast<const uint4*>(rq + so));
+          if (do_x) xv[do_x ? j : 0] = __ldg(reinterpret_cast<const uint4*>(xq + so));
+          if (do_r) rv[do_r ? j : 0] = __ldg(reinterpret_cast<const uint4*>(rq + so));
         }
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
+      for (int j = 0; j < kRows; ++j) {
         const int r = r0 + 8 * j;
         if (r < n_rows) {
           const size_t po = (size_t)(mt * 128 + r) * row_bytes + (size_t)c * 16;
-          if (do_x) __stcs(reinterpret_cast<uint4*>(xq_pad + po), xv[j]);
+          if (do_x) __stcs(reinterpret_cast<uint4*>(xq_pad + po), xv[do_x ? j : 0]);
           if (do_r) {
-            uint4 v = rv[j];
+            uint4 v = rv[do_r ? j : 0];
             v.x = (v.x & m0) ^ 0x88888888u; v.y = (v.y & m1) ^ 0x88888888u;
             v.z = (v.z & m2) ^ 0x88888888u; v.w = (v.w & m3) ^ 0x88888888u;
             __stcs(reinterpret_cast<uint4*>(rq_pad + po), v);
@@ -1043,46 +1046,72 @@ rac_dispatch_kernel(int H, int parts, const uint8_t* __restrict__ mask, const in
     __syncthreads();                                  // the previous slab has been written out
     for (int i = threadIdx.x; i < nk * 32; i += blockDim.x) {
       if (do_x) reinterpret_cast<uint4*>(atoms[0])[i] = make_uint4(0, 0, 0, 0);
-      if (do_r) reinterpret_cast<uint4*>(atoms[1])[i] = make_uint4(0, 0, 0, 0);
+      if (do_r) reinterpret_cast<uint4*>(atoms[kParts == 3 ? 1 : 0])[i] = make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
-    // a thread moves 16 bytes = four atoms' worth of one row; consecutive threads take consecutive pieces
+    // a thread moves 16 bytes = four atoms' worth of one row; consecutive threads take consecutive pieces;
+    // at most 128 rows x 8 pieces = four per thread, all fetched before the first is stored
     const int pieces = (nk + 3) >> 2;
-    for (int i = threadIdx.x; i < n_rows * pieces; i += blockDim.x) {
-      const int r = i / pieces, pc = i - r * pieces;
-      const size_t so = (size_t)tok[r] * sf_row + (size_t)(k0 + 4 * pc) * 4;
-      const int dst = (r & 31) * 16 + (r >> 5) * 4;
-      const int n4 = min(4, nk - 4 * pc);
-      const bool wide = n4 == 4 && (sf_row & 15) == 0;   // else: word loads (row tails, rows that are not 16-byte aligned)
-      if (do_x) {
-        uint32_t w[4] = {0, 0, 0, 0};
-        if (wide) {
-          const uint4 v = __ldg(reinterpret_cast<const uint4*>(xsf + so));
-          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-        } else {
-          for (int j = 0; j < n4; ++j) w[j] = __ldg(reinterpret_cast<const uint32_t*>(xsf + so) + j);
-        }
-        for (int j = 0; j < n4; ++j) *reinterpret_cast<uint32_t*>(&atoms[0][(4 * pc + j) * 512 + dst]) = w[j];
+    const int n_items = n_rows * pieces;
+    auto fetch = [&](const uint8_t* src, size_t so, int n4, bool wide) -> uint4 {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (wide) {
+        v = __ldg(reinterpret_cast<const uint4*>(src + so));
+      } else {                                           // word loads (row tails, rows that are not 16-byte aligned)
+        const uint32_t* s = reinterpret_cast<const uint32_t*>(src + so);
+        if (n4 > 0) v.x = __ldg(s);
+        if (n4 > 1) v.y = __ldg(s + 1);
+        if (n4 > 2) v.z = __ldg(s + 2);
+        if (n4 > 3) v.w = __ldg(s + 3);
       }
-      if (do_r) {
-        uint32_t w[4] = {0, 0, 0, 0};
-        if (wide) {
-          const uint4 v = __ldg(reinterpret_cast<const uint4*>(rsf + so));
-          w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-        } else {
-          for (int j = 0; j < n4; ++j) w[j] = __ldg(reinterpret_cast<const uint32_t*>(rsf + so) + j);
-        }
-        for (int j = 0; j < n4; ++j) *reinterpret_cast<uint32_t*>(&atoms[1][(4 * pc + j) * 512 + dst]) = w[j];
+      return v;
+    };
+    auto put = [&](uint8_t* atom, int pc, int dst, int n4, const uint4& v) {
+      uint32_t* a = reinterpret_cast<uint32_t*>(atom + (4 * pc) * 512 + dst);
+      if (n4 > 0) a[0] = v.x;
+      if (n4 > 1) a[128] = v.y;
+      if (n4 > 2) a[256] = v.z;
+      if (n4 > 3) a[384] = v.w;
+    };
+    uint4 xw[do_x ? 4 : 1], rw[do_r ? 4 : 1];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = threadIdx.x + u * 256;
+      if (i < n_items) {
+        const int r = i / pieces, pc = i - r * pieces;
+        const size_t so = (size_t)tok[r] * sf_row + (size_t)(k0 + 4 * pc) * 4;
+        const int n4 = min(4, nk - 4 * pc);
+        const bool wide = n4 == 4 && (sf_row & 15) == 0;
+        if (do_x) xw[do_x ? u : 0] = fetch(xsf, so, n4, wide);
+        if (do_r) rw[do_r ? u : 0] = fetch(rsf, so, n4, wide);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = threadIdx.x + u * 256;
+      if (i < n_items) {
+        const int r = i / pieces, pc = i - r * pieces;
+        const int dst = (r & 31) * 16 + (r >> 5) * 4;
+        const int n4 = min(4, nk - 4 * pc);
+        if (do_x) put(atoms[0], pc, dst, n4, xw[do_x ? u : 0]);
+        if (do_r) put(atoms[kParts == 3 ? 1 : 0], pc, dst, n4, rw[do_r ? u : 0]);
       }
     }
     __syncthreads();
     const size_t ao = ((size_t)mt * kt_count + k0) * 512u;
     for (int i = threadIdx.x; i < nk * 32; i += blockDim.x) {
       if (do_x) __stcs(reinterpret_cast<uint4*>(xsf_tiled + ao) + i, reinterpret_cast<const uint4*>(atoms[0])[i]);
-      if (do_r) __stcs(reinterpret_cast<uint4*>(rsf_tiled + ao) + i, reinterpret_cast<const uint4*>(atoms[1])[i]);
+      if (do_r) __stcs(reinterpret_cast<uint4*>(rsf_tiled + ao) + i, reinterpret_cast<const uint4*>(atoms[kParts == 3 ? 1 : 0])[i]);
     }
   }
 }
+
+template __global__ void rac_dispatch_kernel<1>(int, const uint8_t*, const int32_t*, const int32_t*, const int32_t*, const uint8_t*,
+                                                const uint8_t*, const uint8_t*, const uint8_t*, uint8_t*, uint8_t*, uint8_t*, uint8_t*);
+template __global__ void rac_dispatch_kernel<2>(int, const uint8_t*, const int32_t*, const int32_t*, const int32_t*, const uint8_t*,
+                                                const uint8_t*, const uint8_t*, const uint8_t*, uint8_t*, uint8_t*, uint8_t*, uint8_t*);
+template __global__ void rac_dispatch_kernel<3>(int, const uint8_t*, const int32_t*, const int32_t*, const int32_t*, const uint8_t*,
+                                                const uint8_t*, const uint8_t*, const uint8_t*, uint8_t*, uint8_t*, uint8_t*, uint8_t*);
 
 // Clear (in place) the codes of unselected channels of a padded [rows, C/2]
 // code matrix; one thread per 16 bytes (32 channels).  A thread keeps its column

@@ -861,7 +861,15 @@ rank_select_kernel(const unsigned long long* __restrict__ score_keys, int C, int
   pdl_sync();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* sc = reinterpret_cast<unsigned long long*>(smem_raw);
-  for (int i = threadIdx.x; i < C; i += blockDim.x) sc[i] = score_keys[i];
+  for (int i0 = threadIdx.x; i0 < C; i0 += 8 * 256) {      // eight loads in flight per thread, then the stores
+    unsigned long long k[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (i0 + u * 256 < C) k[u] = __ldcg(score_keys + i0 + u * 256);
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (i0 + u * 256 < C) sc[i0 + u * 256] = k[u];
+  }
   __syncthreads();
   const int j = blockIdx.x * 16 + (threadIdx.x >> 4);
   const int sub = threadIdx.x & 15;
@@ -1129,11 +1137,18 @@ mask_codes_kernel(uint8_t* __restrict__ codes, const int* __restrict__ n_rows_pt
     const uint8_t* m = mask + c * 32;
     const uint32_t m0 = nibble_mask8(m), m1 = nibble_mask8(m + 8), m2 = nibble_mask8(m + 16), m3 = nibble_mask8(m + 24);
     if ((m0 & m1 & m2 & m3) == 0xFFFFFFFFu) return;          // every channel of this chunk is selected
-    for (int r = blockIdx.x * rows_per_pass + rl; r < n_rows; r += gridDim.x * rows_per_pass) {
-      uint4* p = reinterpret_cast<uint4*>(codes + (size_t)r * (C >> 1)) + c;
-      uint4 v = *p;
-      v.x &= m0; v.y &= m1; v.z &= m2; v.w &= m3;
-      *p = v;
+    const int step = gridDim.x * rows_per_pass;
+    for (int r0 = blockIdx.x * rows_per_pass + rl; r0 < n_rows; r0 += 8 * step) {   // eight rows in flight per thread
+      uint4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (r0 + u * step < n_rows) v[u] = __ldcg(reinterpret_cast<const uint4*>(codes + (size_t)(r0 + u * step) * (C >> 1)) + c);
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (r0 + u * step < n_rows) {
+          v[u].x &= m0; v[u].y &= m1; v[u].z &= m2; v[u].w &= m3;
+          reinterpret_cast<uint4*>(codes + (size_t)(r0 + u * step) * (C >> 1))[c] = v[u];
+        }
     }
     return;
   }

@@ -474,6 +474,17 @@ def run_ours(args):
                 "traffic": None, "ms": g1_ms,
                 "gemm2": {"ms": g2_ms, "achieved": f_alg2 / (g2_ms * 1e-3) / 1e12, "frac": f_alg2 / (g2_ms * 1e-3) / 1e12 / fp4_peak},
                 "frac_of_nominal_9pf": ach / 9000.0}
+    # what the tensor pipe executes for those algorithmic flops: the masked residual product runs at full K
+    # (2 MMAs per K step at a compensated site) and every expert's rows are padded to whole 128-row tiles
+    res_x = B.moe_w4a4_rac(x_d, lg_d, gw13, gw2, topk, n13, n2, a2, workspace=ws, out=out_d, export=True)
+    offs = res_x["offsets"].cpu().numpy().astype("int64")
+    counts = offs[1:] - offs[:-1]
+    padded_rows = int((((counts + 127) // 128) * 128).sum())
+    f_exec1 = 2.0 * padded_rows * H * 2 * I * (2.0 if n13 > 0 else 1.0)
+    roofline["executed"] = {"tflops": f_exec1 / (g1_ms * 1e-3) / 1e12, "frac_of_peak": f_exec1 / (g1_ms * 1e-3) / 1e12 / fp4_peak,
+                            "padded_rows": padded_rows, "dispatched_rows": int(A),
+                            "note": "MMAs issued (residual product at full K, padding rows included); not a roofline claim"}
+    del res_x
     # dram__bytes_read.sum + dram__bytes_write.sum of one GEMM-1 launch: taken from the ncu summary of this
     # workload, and only while the kernel's sources still are the ones that capture ran (else null)
     if args.workload == "prefill" and args.variant == "both":

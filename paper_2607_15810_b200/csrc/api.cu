@@ -114,10 +114,10 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // ------------------------------------------------------------------ workspace
 struct MoeLayout {
-  size_t header, amax, counters13, counters2, expert_total, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
+  size_t header, amax, counters13, keys13, keys2, expert_total, ids, wts, chunk_counts, chunk_base, offsets, tile_prefix, tile_expert, tile_rows;
   size_t perm, pos_pad, row_token, row_weight;
-  size_t partials13, scores13, keys13, keys2, sel13, mask13, xq_tok, xsf_tok, rq_tok, rsf_tok, xq_pad, xsf, rq_pad, rsf;
-  size_t hq_pad, hsf, r2q_pad, r2sf, partials2, scores2, sel2, mask2, y_pad, dec;
+  size_t partials13, scores13, sel13, mask13, xq_tok, xsf_tok, rq_tok, rsf_tok, xq_pad, xsf, rq_pad, rsf;
+  size_t hq_pad, hsf, r2q_pad, r2sf, sel2, mask2, y_pad, dec;
   size_t total;
   int n_chunks, m_tiles_max, stats_ctas, rows_per_cta;
 };
@@ -141,7 +141,8 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   L.header = take(kHdrWords * 4);
   L.amax = take((size_t)kAmaxPartsMax * 4);    // the amax word; also the quantizer's scratch in the one-sided modes
   L.counters13 = take((size_t)((H + 31) / 32) * 4);
-  L.counters2 = take((size_t)((I + 31) / 32 + 1) * 4);
+  L.keys13 = take((size_t)H * 8);                  // integer column scores of site 13 (small batches), zeroed with the header
+  L.keys2 = take((size_t)I * 8);                   // zeroed with the header: the first projection's epilogue adds to it
   L.expert_total = take((size_t)Ee * 4);           // zeroed with the header: the routing kernel adds to it
   L.ids = take((size_t)A * 4);
   L.wts = take((size_t)A * 4);
@@ -157,7 +158,6 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
   L.row_weight = take(pad_rows * 4);
   L.partials13 = take((size_t)L.stats_ctas * H * 4);
   L.scores13 = take((size_t)H * 8 * kScoreSlices);
-  L.keys13 = take((size_t)H * 8);
   L.sel13 = take((size_t)H * 4);
   L.mask13 = take((size_t)H);
   L.xq_tok = take((size_t)T * (H / 2));
@@ -173,9 +173,6 @@ MoeLayout moe_layout(int T, int H, int I, int E, int topk, int N) {
     L.hsf = take((size_t)L.m_tiles_max * (I / 64) * 512);
     L.r2q_pad = take(pad_rows * (I / 2));
     L.r2sf = take((size_t)L.m_tiles_max * (I / 64) * 512);
-    L.partials2 = take((size_t)L.m_tiles_max * 4 * I * 4);
-    L.scores2 = take((size_t)I * 8 * kScoreSlices);
-    L.keys2 = take((size_t)I * 8);
     L.sel2 = take((size_t)I * 4);
     L.mask2 = take((size_t)I);
     L.y_pad = take(pad_rows * (size_t)H * 2);
@@ -269,10 +266,9 @@ int gemm_cta_group_for(int64_t rows, int experts) {
   return rows >= (int64_t)1024 * (experts > 0 ? experts : 1) ? 2 : 1;
 }
 
-quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
-                        int n_sel, double* slice_sums, unsigned int* counters, unsigned long long* keys,
-                        uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
-  QUADS_CUDA_OK(launch_kernel(score_reduce_kernel, dim3((C + 31) / 32, kScoreSlices), dim3(256), (size_t)(0), st, partials, n_part_ptr, n_part_mul, n_part_fixed, C, slice_sums, counters, keys));
+// Ranking of C order-preserving 64-bit score keys: mask of the n_sel largest (+ their ascending list).
+quads_status run_rank(const unsigned long long* keys, int C, int n_sel, uint8_t* mask, int32_t* sel_export,
+                      cudaStream_t st) {
   QUADS_CUDA_OK(set_max_dynamic_smem<rank_select_kernel>(128 * 1024));
   QUADS_CUDA_OK(launch_kernel(rank_select_kernel, dim3((C + 15) / 16), dim3(256), (size_t)((size_t)C * 8), st, keys, C, n_sel, mask));
   if (sel_export) {
@@ -280,6 +276,13 @@ quads_status run_select(const float* partials, const int* n_part_ptr, int n_part
   }
   QUADS_CUDA_OK(cudaGetLastError());
   return QUADS_OK;
+}
+
+quads_status run_select(const float* partials, const int* n_part_ptr, int n_part_mul, int n_part_fixed, int C,
+                        int n_sel, double* slice_sums, unsigned int* counters, unsigned long long* keys,
+                        uint8_t* mask, int32_t* sel_export, cudaStream_t st) {
+  QUADS_CUDA_OK(launch_kernel(score_reduce_kernel, dim3((C + 31) / 32, kScoreSlices), dim3(256), (size_t)(0), st, partials, n_part_ptr, n_part_mul, n_part_fixed, C, slice_sums, counters, keys));
+  return run_rank(keys, C, n_sel, mask, sel_export, st);
 }
 
 }  // namespace
@@ -572,7 +575,8 @@ quads_status quads_rac_channel_scores(const void* x, int64_t T, int64_t H, const
   const int block = H / 16 > 256 ? 256 : (int)((H / 16 + 31) / 32 * 32);
   QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(ctas), dim3(block), (size_t)0, st, xp, (int)T, (int)H, gs_in, amax_bits,
                               (unsigned int*)nullptr, status_word, (float*)nullptr, rpc, 1, partials, (uint8_t*)nullptr,
-                              (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr));
+                              (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr, (uint8_t*)nullptr,
+                              (unsigned long long*)nullptr, 0, 0));
   // the order-preserving 64-bit keys of non-negative scores are the scores' own bit patterns
   QUADS_CUDA_OK(launch_kernel(score_reduce_kernel, dim3((unsigned)((H + 31) / 32), kScoreSlices), dim3(256), (size_t)0, st,
                               (const float*)partials, (const int*)nullptr, 1, ctas, (int)H, slices, counters,
@@ -816,6 +820,7 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   trace_mark("amax", st);
   // ---- site 13: quantize (+ residual + statistics), selection, dispatch scatter
   const int nsel13 = a->rac_nsel_13;
+  const bool totals13 = (int64_t)L.stats_ctas * H <= ((int64_t)1 << 18);
   uint8_t* mask13 = P(L.mask13);
   {
     const uint16_t* xp = x;
@@ -824,19 +829,30 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     unsigned int* arrivals = fused_amax ? reinterpret_cast<unsigned int*>(header + kHdrArrivals) : nullptr;
     int32_t* status_word = header + kHdrStatus;
     float* gs_store = a->a13_gs_out;
-    float* partials = reinterpret_cast<float*>(P(L.partials13));
+    // Column scores of site 13: integer totals added by every CTA when there are few of them (the
+    // selection is then one ranking kernel; decode-sized batches), else one partial row per CTA and a
+    // reduction kernel (586 x 2048 integer reductions at the end of the kernel cost 20 us, the
+    // reduction kernel 9)
+    float* partials = totals13 ? nullptr : reinterpret_cast<float*>(P(L.partials13));
+    unsigned long long* totals = totals13 ? reinterpret_cast<unsigned long long*>(P(L.keys13)) : nullptr;
+    // a CTA's partial sum covers rows_per_cta rows (< rows * 2^18 in units of the squared scale); the
+    // stats_ctas partial sums of a column must fit 62 bits together
+    int cap_bits = 18, ctas_log2 = 0;
+    while ((1 << (cap_bits - 18)) < rows_per_cta) ++cap_bits;
+    while ((1 << ctas_log2) < L.stats_ctas) ++ctas_log2;
+    int score_bits = std::max(0, std::min(26, 62 - cap_bits - ctas_log2));
     uint8_t *xq_tok = P(L.xq_tok), *xsf_tok = P(L.xsf_tok), *rq_tok = P(L.rq_tok), *rsf_tok = P(L.rsf_tok);
     uint8_t *xq_exp = a->xq, *xsf_exp = a->xsf;
     if (fused_amax) {
       void* args[] = {&xp, &Tt, &Hh, &gs13, &amax_bits, &arrivals, &status_word, &gs_store, &rows_per_cta, &with_res,
-                      &partials, &xq_tok, &xsf_tok, &rq_tok, &rsf_tok, &xq_exp, &xsf_exp};
+                      &partials, &xq_tok, &xsf_tok, &rq_tok, &rsf_tok, &xq_exp, &xsf_exp, &totals, &score_bits, &cap_bits};
       QUADS_CUDA_OK(cudaLaunchCooperativeKernel(reinterpret_cast<void*>(rac_quant_kernel), dim3(L.stats_ctas),
                                                 dim3(rq_block), args, 0, st));
       note_launch();
     } else {
       QUADS_CUDA_OK(launch_kernel(rac_quant_kernel, dim3(L.stats_ctas), dim3(rq_block), (size_t)(0), st, xp, Tt, Hh, gs13,
                                   amax_bits, arrivals, status_word, gs_store, rows_per_cta, with_res, partials, xq_tok,
-                                  xsf_tok, rq_tok, rsf_tok, xq_exp, xsf_exp));
+                                  xsf_tok, rq_tok, rsf_tok, xq_exp, xsf_exp, totals, score_bits, cap_bits));
     }
   }
   trace_mark("rac_stats", st);
@@ -860,9 +876,12 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
     }
   }
   if (nsel13 > 0) {
-    s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
-                   reinterpret_cast<double*>(P(L.scores13)), reinterpret_cast<unsigned int*>(P(L.counters13)),
-                   reinterpret_cast<unsigned long long*>(P(L.keys13)), mask13, a->sel13, st);
+    if (totals13)
+      s = run_rank(reinterpret_cast<unsigned long long*>(P(L.keys13)), H, nsel13, mask13, a->sel13, st);
+    else
+      s = run_select(reinterpret_cast<float*>(P(L.partials13)), nullptr, 1, L.stats_ctas, H, nsel13,
+                     reinterpret_cast<double*>(P(L.scores13)), reinterpret_cast<unsigned int*>(P(L.counters13)),
+                     reinterpret_cast<unsigned long long*>(P(L.keys13)), mask13, a->sel13, st);
     if (s != QUADS_OK) return s;
   }
   trace_mark("select13", st);
@@ -928,7 +947,14 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   g.h_gs = a->a2_gs;
   g.resid2 = a->rac_nsel_2 > 0 || a->r2q || a->r2sf;
   g.hq_pad = P(L.hq_pad); g.hsf_tiled = P(L.hsf); g.r2q_pad = P(L.r2q_pad); g.r2sf_tiled = P(L.r2sf);
-  g.partials2 = reinterpret_cast<float*>(P(L.partials2));
+  g.keys2 = reinterpret_cast<unsigned long long*>(P(L.keys2));
+  {
+    // fractional bits of the integer column scores: a partial sum stays below 2^23 (in units of the
+    // squared scale), there are at most 4 per row tile, and their total must fit 62 bits
+    int rows_log2 = 0;
+    while (((int64_t)1 << rows_log2) < (int64_t)L.m_tiles_max * 4) ++rows_log2;
+    g.score_bits = std::max(0, std::min(26, 62 - 23 - rows_log2));
+  }
   g.h_export = static_cast<uint16_t*>(a->h_bf16);
   const bool timing = g_timers.enabled && g_timers.created;
   if (timing) QUADS_CUDA_OK(cudaEventRecord(g_timers.ev[0], st));
@@ -942,9 +968,8 @@ quads_status quads_moe_w4a4_rac(const quads_moe_args* a, void* cuda_stream) {
   const int nsel2 = a->rac_nsel_2;
   uint8_t* mask2 = P(L.mask2);
   if (nsel2 > 0) {
-    s = run_select(g.partials2, header + kHdrMTiles, 4 /* one partial row per tile and lane quadrant */, 0, I, nsel2,
-                   reinterpret_cast<double*>(P(L.scores2)), reinterpret_cast<unsigned int*>(P(L.counters2)),
-                   reinterpret_cast<unsigned long long*>(P(L.keys2)), mask2, a->sel2, st);
+    // the scores are complete when the first projection ends (integer totals): ranking only
+    s = run_rank(g.keys2, I, nsel2, mask2, a->sel2, st);
     if (s != QUADS_OK) return s;
     QUADS_CUDA_OK(launch_kernel(mask_codes_kernel, dim3(di.sm_count * 8), dim3(256), (size_t)(0), st, P(L.r2q_pad), header + kHdrPaddedRows, I, mask2));
   } else if (a->r2q) {

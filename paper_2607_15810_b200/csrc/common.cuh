@@ -234,6 +234,19 @@ __device__ __forceinline__ void store_y_rows(const float* acc, float scale, uint
   }
 }
 
+// One partial column score (a float32 sum of squared residuals, >= 0) as a fixed-point integer with
+// `bits` fractional bits in units of gs^2, capped at 2^(cap_bits + bits): a residual is at most half a
+// quantization step, 448 gs, so a sum over n rows stays below n * 2^18 gs^2 (cap_bits = 18 + log2 n).
+// Added to the column's total with an integer reduction, whose result does not depend on the order of
+// the additions.
+__device__ __forceinline__ void add_score(unsigned long long* total, float partial, float gs, int bits, int cap_bits = 23) {
+  const float u = __fdiv_rn(__fdiv_rn(partial, gs), gs);
+  const float cap = __uint_as_float((uint32_t)(127 + cap_bits + bits) << 23);
+  const float v = fminf(u * __uint_as_float((uint32_t)(127 + bits) << 23), cap);
+  const unsigned long long q = __float2ull_rd(v);
+  if (q) asm volatile("red.global.add.u64 [%0], %1;" ::"l"(total), "l"(q) : "memory");
+}
+
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));

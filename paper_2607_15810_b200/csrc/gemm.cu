@@ -435,7 +435,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p, const CUtensorMap
             const float cs = warp_colsum16(r, lane);
             if ((lane & 1) == 0) {
               const int col = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-              p.partials2[(size_t)(mt * 4 + q) * I + f0 + 16 * c + col] = cs;
+              add_score(p.keys2 + f0 + 16 * c + col, cs, qc.gs, p.score_bits);
             }
           }
         }

@@ -402,17 +402,14 @@ gemm_swapped_kernel(const GemmParams p, const __grid_constant__ CUtensorMap tm_x
                                   r[4 * i + 3] * r[4 * i + 3]);
           }
         }
-        // (3) column scores of the residual: sum over the chunk's tokens in token order -> partial
-        // row (slot, chunk); the slot's first chunk also clears the rows of its absent chunks.
+        // (3) column scores of the residual: sum over the chunk's tokens in token order, then into the
+        // column's integer total
         if (p.resid2) {
           epi_barrier();
           if (etid < 128) {
             float sacc = 0.f;
             for (int tt = 0; tt < n_rows; ++tt) sacc += rs[tt * 128 + etid];
-            p.partials2[(size_t)(mt * 4 + c) * I + ft * 128 + etid] = sacc;
-            if (c == 0)
-              for (int cc = ((int)tab_rows[mt] + kChunk - 1) / kChunk; cc < 4; ++cc)
-                p.partials2[(size_t)(mt * 4 + cc) * I + ft * 128 + etid] = 0.f;
+            add_score(p.keys2 + ft * 128 + etid, sacc, p.h_gs[0], p.score_bits);
           }
         }
       }

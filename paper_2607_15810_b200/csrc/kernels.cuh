@@ -40,7 +40,9 @@ __global__ void dequantize_kernel(const uint8_t* q, const uint8_t* sf, const flo
 __global__ void rac_quant_kernel(const uint16_t* x, int T, int H, const float* gs_in, uint32_t* amax_bits,
                                  unsigned int* grid_arrivals, int32_t* status,
                                  float* gs_store, int rows_per_cta, int with_residual, float* partials, uint8_t* xq,
-                                 uint8_t* xsf, uint8_t* rq, uint8_t* rsf, uint8_t* xq_exp, uint8_t* xsf_exp);
+                                 uint8_t* xsf, uint8_t* rq, uint8_t* rsf, uint8_t* xq_exp, uint8_t* xsf_exp,
+                                 unsigned long long* score_totals /* or NULL: partial rows */, int score_bits,
+                                 int cap_bits);
 constexpr int kScoreSlices = 16;
 __global__ void score_reduce_kernel(const float* partials, const int* n_part_ptr, int n_part_mul,
                                     int n_part_fixed, int C, double* slice_sums, unsigned int* counters,
@@ -118,7 +120,12 @@ struct GemmParams {
   const float* h_gs;     // per-tensor scale of h
   int resid2;            // 1: also emit the residual of h and its column statistics
   uint8_t* hq_pad; uint8_t* hsf_tiled; uint8_t* r2q_pad; uint8_t* r2sf_tiled;
-  float* partials2;      // [4 * m_tiles, n_out]
+  // column scores of the residual of h (Eq. channel-score), accumulated as integers so that the sum does
+  // not depend on the order of arrival: every partial sum of squares (one per tile, lane quadrant and
+  // column) is divided by the square of h's per-tensor scale, multiplied by 2^score_bits, rounded down
+  // and added with a 64-bit integer reduction; the totals are the selection's order-preserving keys
+  unsigned long long* keys2;   // [n_out], zero on entry
+  int score_bits;
   uint16_t* h_export;    // optional bf16 [A, n_out] in dispatch order
   const int32_t* tile_prefix;
   const int32_t* offsets;

@@ -712,7 +712,8 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
                  float* __restrict__ gs_store, int rows_per_cta,
                  int with_residual, float* __restrict__ partials, uint8_t* __restrict__ xq,
                  uint8_t* __restrict__ xsf, uint8_t* __restrict__ rq, uint8_t* __restrict__ rsf,
-                 uint8_t* __restrict__ xq_exp, uint8_t* __restrict__ xsf_exp) {
+                 uint8_t* __restrict__ xq_exp, uint8_t* __restrict__ xsf_exp,
+                 unsigned long long* __restrict__ score_totals, int score_bits, int cap_bits) {
   pdl_sync();
   const int k16 = H >> 4;
   const int r0 = blockIdx.x * rows_per_cta;
@@ -798,7 +799,11 @@ rac_quant_kernel(const uint16_t* __restrict__ x, int T, int H, const float* __re
         }
       }
     }
-    if (with_residual) {
+    if (with_residual && score_totals) {
+      // integer totals per channel (zero on entry): complete when the kernel ends, whatever the order
+#pragma unroll
+      for (int i = 0; i < 16; ++i) add_score(score_totals + kb * 16 + i, acc[i], gs, score_bits, cap_bits);
+    } else if (with_residual) {
       float4* dst = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * H + kb * 16);
       dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
       dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);

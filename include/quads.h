@@ -198,6 +198,10 @@ quads_status quads_fake_quant_weights_noalloc(const void* w, int64_t n_tensors, 
  * id), weights = softmax over all experts restricted to the chosen ones
  * (renormalised when `renormalize`), h = silu(W1 x) * (W3 x) rounded to bf16,
  * requantized with `a2_gs`, out = sum_k weight_k * W2 h~.
+ * The output is reproducible bit for bit: every floating-point sum runs in a
+ * fixed order, and the channel scores that cross CTAs are added as 64-bit
+ * integers (partial sum of squares / scale^2, at most 26 fractional bits), so
+ * the selection does not depend on the order in which CTAs finish.
  *
  * Dense mode (I == 0): one projection out[T, N] = W X~ with E = topk = 1, the
  * weight in w13_*, no routing, no SwiGLU ("single dense W4A4+RAC GEMM").  With
